@@ -1,0 +1,288 @@
+// NVFP4 CPU oracle -- TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT.
+// See nvfp4_oracle.h.  Plain C++17, no CUDA, no code shared with the GPU path.
+// Build: g++ -O2 -std=c++17 -ffp-contract=off -fPIC -shared -pthread
+//
+// Readings taken where the paper is silent (all listed in the design notes):
+//   * the block scale is amax * ((1/6)/g) rounded to unsigned E4M3 (nearest,
+//     ties to even, saturating at 448): "block amax mapped to 6";
+//   * elements are divided by the *decoded* scale, clamped to 6, then rounded;
+//   * RtN ties go to the code with an even mantissa bit;
+//   * SR acts on the magnitude and spends one random byte per element.
+#include "nvfp4_oracle.h"
+
+#include <cmath>
+#include <cstring>
+#include <functional>
+#include <thread>
+#include <vector>
+
+namespace {
+
+// Section 3: the eight E2M1 magnitudes, index = 3-bit code ee|m.
+const float kGrid[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f};
+
+void parallel_rows(int64_t rows, int nthreads, const std::function<void(int64_t, int64_t)>& fn) {
+  if (nthreads <= 1 || rows < 2) { fn(0, rows); return; }
+  if (nthreads > rows) nthreads = (int)rows;
+  std::vector<std::thread> pool;
+  int64_t per = (rows + nthreads - 1) / nthreads;
+  for (int t = 0; t < nthreads; ++t) {
+    int64_t lo = t * per, hi = lo + per < rows ? lo + per : rows;
+    if (lo >= hi) break;
+    pool.emplace_back(fn, lo, hi);
+  }
+  for (auto& th : pool) th.join();
+}
+
+inline float code_value(uint8_t nib) {            // signed value of a 4-bit code
+  float m = kGrid[nib & 7];
+  return (nib & 8) ? -m : m;
+}
+
+}  // namespace
+
+extern "C" {
+
+float nvfp4o_e2m1_decode(uint8_t code) {
+  // Section 3: 1 sign, 2 exponent, 1 mantissa bit; exponent bias 1.
+  int s = (code >> 3) & 1, e = (code >> 1) & 3, m = code & 1;
+  float mag = (e == 0) ? 0.5f * (float)m                       // subnormal: m * 2^(1-1) / 2
+                       : std::ldexp(1.0f + 0.5f * (float)m, e - 1);
+  return s ? -mag : mag;
+}
+
+float nvfp4o_e4m3_decode(uint8_t code) {
+  int e = (code >> 3) & 15, m = code & 7;
+  if (e == 15 && m == 7) return NAN;                           // the single NaN pattern
+  if (e == 0) return std::ldexp((float)m, -9);                 // subnormal: m/8 * 2^-6
+  return std::ldexp(1.0f + (float)m / 8.0f, e - 7);
+}
+
+uint8_t nvfp4o_e4m3_encode(float v) {
+  if (std::isnan(v)) return 0x7F;
+  if (!(v > 0.0f)) return 0;                                   // zero (sign unused; negatives never occur)
+  if (v > 448.0f) return 0x7E;                                 // saturate to the largest finite value
+  // Quantum of the binade that holds v: 2^(e-3) for normals, 2^-9 below 2^-6.
+  int e;
+  (void)std::frexp(v, &e);                                     // v = f * 2^e, f in [0.5,1)
+  int ue = e - 1;                                              // floor(log2 v)
+  if (ue < -6) ue = -6;
+  float quantum = std::ldexp(1.0f, ue - 3);
+  float q = v / quantum;                                       // exact (power of two)
+  float r = std::nearbyintf(q);                                // default mode: nearest, ties to even
+  float val = r * quantum;                                     // exact
+  if (val > 448.0f) return 0x7E;
+  if (val == 0.0f) return 0;
+  // Turn the rounded value back into bits.
+  (void)std::frexp(val, &e);
+  ue = e - 1;
+  if (ue < -6) return (uint8_t)std::lrintf(val * 512.0f);      // subnormal mantissa m = val / 2^-9
+  int mant = (int)std::lrintf((val / std::ldexp(1.0f, ue) - 1.0f) * 8.0f);
+  return (uint8_t)(((ue + 7) << 3) | mant);
+}
+
+void nvfp4o_philox4x32_10(const uint32_t key[2], const uint32_t ctr[4], uint32_t out[4]) {
+  const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;           // round multipliers
+  const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;           // Weyl key increments
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    uint64_t p0 = (uint64_t)M0 * c0, p1 = (uint64_t)M1 * c2;
+    uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+    uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+    uint32_t n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += W0; k1 += W1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+void nvfp4o_block_random_bytes(uint64_t seed, uint64_t offset, uint64_t block, uint8_t out[16]) {
+  uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t ctr[4] = {(uint32_t)block, (uint32_t)(block >> 32), (uint32_t)offset, (uint32_t)(offset >> 32)};
+  uint32_t w[4];
+  nvfp4o_philox4x32_10(key, ctr, w);
+  for (int j = 0; j < 16; ++j) out[j] = (uint8_t)(w[j / 4] >> (8 * (j % 4)));
+}
+
+uint8_t nvfp4o_round_rtn(float y) {
+  // Closest grid magnitude; on an exact tie keep the code whose mantissa bit is 0.
+  int best = 0;
+  double best_d = std::fabs((double)y - (double)kGrid[0]);
+  for (int c = 1; c < 8; ++c) {
+    double d = std::fabs((double)y - (double)kGrid[c]);
+    if (d < best_d || (d == best_d && (c & 1) == 0)) { best = c; best_d = d; }
+  }
+  return (uint8_t)best;
+}
+
+uint8_t nvfp4o_round_sr(float y, uint8_t u8) {
+  // Grid spacing around y, then round t = y/spacing up with probability frac(t).
+  float delta = (y < 2.0f) ? 0.5f : (y < 4.0f) ? 1.0f : 2.0f;
+  float t = y / delta;                                         // exact
+  float lo = std::floor(t);
+  float f = t - lo;                                            // exact
+  float u = ((float)u8 + 0.5f) / 256.0f;                       // exact, in (0,1)
+  float val = (lo + ((u < f) ? 1.0f : 0.0f)) * delta;          // a grid value
+  for (int c = 0; c < 8; ++c) if (kGrid[c] == val) return (uint8_t)c;
+  return 7;                                                    // unreachable for y in [0,6]
+}
+
+void nvfp4o_quantize(const float* x, int64_t Rq, int64_t Kq, float g, int mode,
+                     uint64_t seed, uint64_t offset,
+                     uint8_t* codes, uint8_t* scales, int nthreads) {
+  const int64_t nkb = Kq / 16;
+  const float c = (1.0f / 6.0f) / g;                           // once per call: two fp32 divisions
+  parallel_rows(Rq, nthreads, [=](int64_t r0, int64_t r1) {
+    for (int64_t r = r0; r < r1; ++r) {
+      for (int64_t kb = 0; kb < nkb; ++kb) {
+        const float* xb = x + r * Kq + kb * 16;
+        float amax = 0.0f;
+        for (int j = 0; j < 16; ++j) { float a = std::fabs(xb[j]); if (a > amax) amax = a; }
+        float s_f = amax * c;                                  // amax mapped to 6
+        uint8_t s_q = nvfp4o_e4m3_encode(s_f);
+        float s_d = nvfp4o_e4m3_decode(s_q);
+        float d = s_d * g;
+        float inv = (s_q == 0) ? 0.0f : 1.0f / d;              // one division per block
+        uint8_t rnd[16];
+        if (mode == 1) nvfp4o_block_random_bytes(seed, offset, (uint64_t)(r * nkb + kb), rnd);
+        uint8_t nib[16];
+        for (int j = 0; j < 16; ++j) {
+          float y = std::fabs(xb[j]) * inv;
+          y = (y < 6.0f) ? y : 6.0f;                           // clamp (also maps NaN to 6)
+          uint8_t m = (mode == 1) ? nvfp4o_round_sr(y, rnd[j]) : nvfp4o_round_rtn(y);
+          nib[j] = (uint8_t)((std::signbit(xb[j]) ? 8 : 0) | m);
+        }
+        uint8_t* cb = codes + (r * Kq + kb * 16) / 2;
+        for (int j = 0; j < 8; ++j) cb[j] = (uint8_t)(nib[2 * j] | (nib[2 * j + 1] << 4));
+        scales[r * nkb + kb] = s_q;
+      }
+    }
+  });
+}
+
+void nvfp4o_quantize_transposed(const float* x, int64_t rows, int64_t cols, float g, int mode,
+                                uint64_t seed, uint64_t offset,
+                                uint8_t* codes, uint8_t* scales, int nthreads) {
+  std::vector<float> xt((size_t)rows * (size_t)cols);
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t c = 0; c < cols; ++c) xt[(size_t)c * rows + r] = x[(size_t)r * cols + c];
+  nvfp4o_quantize(xt.data(), cols, rows, g, mode, seed, offset, codes, scales, nthreads);
+}
+
+void nvfp4o_dequantize(const uint8_t* codes, const uint8_t* scales, float g,
+                       int64_t Rq, int64_t Kq, float* out) {
+  const int64_t nkb = Kq / 16;
+  for (int64_t r = 0; r < Rq; ++r)
+    for (int64_t k = 0; k < Kq; ++k) {
+      uint8_t byte = codes[(r * Kq + k) / 2];
+      uint8_t nib = (k & 1) ? (byte >> 4) : (byte & 15);
+      float d = nvfp4o_e4m3_decode(scales[r * nkb + k / 16]) * g;
+      out[r * Kq + k] = code_value(nib) * d;
+    }
+}
+
+float nvfp4o_tensor_amax_scale(const float* x, int64_t n) {
+  float amax = 0.0f;
+  for (int64_t i = 0; i < n; ++i) { float a = std::fabs(x[i]); if (a > amax) amax = a; }
+  return (amax == 0.0f) ? 1.0f : amax / 2688.0f;               // 6 * 448
+}
+
+static void gemm_one(const uint8_t* a_codes, const uint8_t* a_sf, const uint8_t* b_codes,
+                     const uint8_t* b_sf, int64_t K, int64_t i, int64_t j,
+                     double* acc_out, double* abs_out) {
+  const int64_t nkb = K / 16;
+  double acc = 0.0, aabs = 0.0;
+  for (int64_t kb = 0; kb < nkb; ++kb) {
+    double inner = 0.0, inner_abs = 0.0;
+    for (int k = 0; k < 16; ++k) {
+      int64_t kk = kb * 16 + k;
+      uint8_t ab = a_codes[(i * K + kk) / 2], bb = b_codes[(j * K + kk) / 2];
+      double av = code_value((kk & 1) ? (ab >> 4) : (ab & 15));
+      double bv = code_value((kk & 1) ? (bb >> 4) : (bb & 15));
+      inner += av * bv;
+      inner_abs += std::fabs(av * bv);
+    }
+    double s = (double)nvfp4o_e4m3_decode(a_sf[i * nkb + kb]) * (double)nvfp4o_e4m3_decode(b_sf[j * nkb + kb]);
+    acc += s * inner;
+    aabs += s * inner_abs;
+  }
+  *acc_out = acc;
+  *abs_out = aabs;
+}
+
+void nvfp4o_gemm(const uint8_t* a_codes, const uint8_t* a_sf, float ga,
+                 const uint8_t* b_codes, const uint8_t* b_sf, float gb,
+                 int64_t M, int64_t N, int64_t K, float* D, float* T, int nthreads) {
+  const double alpha = (double)ga * (double)gb;
+  parallel_rows(M, nthreads, [=](int64_t i0, int64_t i1) {
+    for (int64_t i = i0; i < i1; ++i)
+      for (int64_t j = 0; j < N; ++j) {
+        double acc, aabs;
+        gemm_one(a_codes, a_sf, b_codes, b_sf, K, i, j, &acc, &aabs);
+        if (D) D[i * N + j] = (float)(alpha * acc);
+        if (T) T[i * N + j] = (float)(std::fabs(alpha) * aabs);
+      }
+  });
+}
+
+void nvfp4o_gemm_sampled(const uint8_t* a_codes, const uint8_t* a_sf, float ga,
+                         const uint8_t* b_codes, const uint8_t* b_sf, float gb,
+                         int64_t M, int64_t N, int64_t K,
+                         const int64_t* ii, const int64_t* jj, int64_t n,
+                         float* D, float* T) {
+  (void)M; (void)N;
+  const double alpha = (double)ga * (double)gb;
+  for (int64_t s = 0; s < n; ++s) {
+    double acc, aabs;
+    gemm_one(a_codes, a_sf, b_codes, b_sf, K, ii[s], jj[s], &acc, &aabs);
+    if (D) D[s] = (float)(alpha * acc);
+    if (T) T[s] = (float)(std::fabs(alpha) * aabs);
+  }
+}
+
+void nvfp4o_gemm_f32acc(const uint8_t* a_codes, const uint8_t* a_sf, float ga,
+                        const uint8_t* b_codes, const uint8_t* b_sf, float gb,
+                        int64_t M, int64_t N, int64_t K, float* D, int nthreads) {
+  const int64_t nkb = K / 16;
+  const float alpha = ga * gb;
+  parallel_rows(M, nthreads, [=](int64_t i0, int64_t i1) {
+    for (int64_t i = i0; i < i1; ++i)
+      for (int64_t j = 0; j < N; ++j) {
+        float acc = 0.0f;
+        for (int64_t kb = 0; kb < nkb; ++kb) {
+          float inner = 0.0f;
+          for (int k = 0; k < 16; ++k) {
+            int64_t kk = kb * 16 + k;
+            uint8_t ab = a_codes[(i * K + kk) / 2], bb = b_codes[(j * K + kk) / 2];
+            inner += code_value((kk & 1) ? (ab >> 4) : (ab & 15)) * code_value((kk & 1) ? (bb >> 4) : (bb & 15));
+          }
+          float s = nvfp4o_e4m3_decode(a_sf[i * nkb + kb]) * nvfp4o_e4m3_decode(b_sf[j * nkb + kb]);
+          acc += s * inner;
+        }
+        D[i * N + j] = alpha * acc;
+      }
+  });
+}
+
+int64_t nvfp4o_sf_swizzled_offset(int64_t r, int64_t kb, int64_t n_kb) {
+  // Tiles of 128 rows x 4 blocks, 512 bytes each, k-tiles contiguous within a
+  // row tile.  Inside a tile, 16-byte groups are indexed by r % 32; each group
+  // holds the four 32-row quarters of the tile, 4 block scales apiece.
+  int64_t k_tiles = (n_kb + 3) / 4;
+  int64_t tile = (r / 128) * k_tiles + kb / 4;
+  return tile * 512 + (r % 32) * 16 + ((r % 128) / 32) * 4 + (kb % 4);
+}
+
+int64_t nvfp4o_sf_swizzled_bytes(int64_t Rq, int64_t n_kb) {
+  return ((Rq + 127) / 128) * ((n_kb + 3) / 4) * 512;
+}
+
+void nvfp4o_sf_swizzle(const uint8_t* linear, int64_t Rq, int64_t n_kb, uint8_t* out) {
+  std::memset(out, 0, (size_t)nvfp4o_sf_swizzled_bytes(Rq, n_kb));
+  for (int64_t r = 0; r < Rq; ++r)
+    for (int64_t kb = 0; kb < n_kb; ++kb)
+      out[nvfp4o_sf_swizzled_offset(r, kb, n_kb)] = linear[r * n_kb + kb];
+}
+
+}  // extern "C"

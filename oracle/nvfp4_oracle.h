@@ -1,0 +1,106 @@
+/*
+ * NVFP4 CPU oracle -- TEST INFRASTRUCTURE, NOT PART OF THE PRODUCT.
+ *
+ * A plain, slow, obviously-correct restatement of the paper's quantizer
+ * (Section 3: E2M1 elements, blocks of 16, one E4M3 scale per block; Section 1
+ * and Eq. 4-6: round-to-nearest and stochastic rounding) and of the three
+ * linear-layer products (Eq. 1-3) as dequantize-then-matmul.  It shares no code
+ * with the CUDA library and must never be linked, imported or called by it.
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * Everything is host memory.  All functions are single IEEE-754 binary32
+ * operations exactly as written (compile with -ffp-contract=off, no fast-math).
+ *
+ * Parity status: every function below is pinned by tests that do not call it
+ * to produce their own expectations (format definitions, enumeration, closed
+ * forms, published known-answer vectors, a library cast).  The paper prints no
+ * worked numeric example, so none of the pins is a value printed by the paper.
+ */
+#ifndef NVFP4_ORACLE_H
+#define NVFP4_ORACLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Section 3: E2M1 = 1 sign, 2 exponent (bias 1), 1 mantissa bit.  `code` is the
+ * 4-bit pattern s|ee|m in the low nibble. */
+float nvfp4o_e2m1_decode(uint8_t code);
+
+/* Section 3 ("E4M3 format for storing scales"), sign bit unused: unsigned E4M3,
+ * bias 7, 3 mantissa bits, subnormals, largest finite 448 (0x7E), no infinity.
+ * Encode rounds to nearest, ties to the even mantissa, and saturates at 448. */
+uint8_t nvfp4o_e4m3_encode(float v);
+float nvfp4o_e4m3_decode(uint8_t code);
+
+/* Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw 2011). */
+void nvfp4o_philox4x32_10(const uint32_t key[2], const uint32_t ctr[4], uint32_t out[4]);
+
+/* The 16 random bytes of block B: counter (B_lo, B_hi, offset_lo, offset_hi),
+ * key (seed_lo, seed_hi); the four output words little-endian give bytes 0..15. */
+void nvfp4o_block_random_bytes(uint64_t seed, uint64_t offset, uint64_t block, uint8_t out[16]);
+
+/* Section 1: RtN maps y in [0,6] to the closest grid magnitude (ties to the
+ * code with an even mantissa bit); SR picks one of the two neighbours with
+ * probability given by the distance, using one random byte.  Both return the
+ * 3-bit magnitude code. */
+uint8_t nvfp4o_round_rtn(float y);
+uint8_t nvfp4o_round_sr(float y, uint8_t u8);
+
+/* Quantize a logical [Rq, Kq] fp32 tensor (row stride Kq) in blocks of 16 along
+ * Kq.  mode 0 = RtN, 1 = SR.  codes: Rq*Kq/2 bytes (element 2i in the low
+ * nibble of byte i); scales: Rq*Kq/16 bytes, linear [Rq, Kq/16].  Kq % 16 == 0.
+ * g is the per-tensor scale (1.0f = none). */
+void nvfp4o_quantize(const float* x, int64_t Rq, int64_t Kq, float g, int mode,
+                     uint64_t seed, uint64_t offset,
+                     uint8_t* codes, uint8_t* scales, int nthreads);
+
+/* Transposed quantization of x[rows, cols]: by definition nvfp4o_quantize
+ * applied to the materialised transpose (Rq = cols, Kq = rows). */
+void nvfp4o_quantize_transposed(const float* x, int64_t rows, int64_t cols, float g, int mode,
+                                uint64_t seed, uint64_t offset,
+                                uint8_t* codes, uint8_t* scales, int nthreads);
+
+/* out[r, k] = decode(code) * decode(scale) * g  (exact in fp32 when g is a
+ * power of two; otherwise one rounding per factor as written). */
+void nvfp4o_dequantize(const uint8_t* codes, const uint8_t* scales, float g,
+                       int64_t Rq, int64_t Kq, float* out);
+
+/* g = amax / (6*448) in one fp32 division, 1.0f when amax == 0. */
+float nvfp4o_tensor_amax_scale(const float* x, int64_t n);
+
+/* D[i,j] = (gA*gB) * sum_kb sA[i,kb]*sB[j,kb] * sum_{k in kb} a[i,k]*b[j,k]
+ * with A[M,K], B[N,K] both K-major, linear scales; double accumulation, result
+ * rounded to fp32.  T[i,j] = the same sum over absolute values (the tolerance
+ * base).  D and/or T may be NULL. */
+void nvfp4o_gemm(const uint8_t* a_codes, const uint8_t* a_sf, float ga,
+                 const uint8_t* b_codes, const uint8_t* b_sf, float gb,
+                 int64_t M, int64_t N, int64_t K, float* D, float* T, int nthreads);
+
+/* Same contraction with every partial sum kept in fp32 (shows how far plain
+ * fp32 accumulation sits from the double result). */
+void nvfp4o_gemm_f32acc(const uint8_t* a_codes, const uint8_t* a_sf, float ga,
+                        const uint8_t* b_codes, const uint8_t* b_sf, float gb,
+                        int64_t M, int64_t N, int64_t K, float* D, int nthreads);
+
+/* The double-accumulated result at n sampled (i,j) positions only. */
+void nvfp4o_gemm_sampled(const uint8_t* a_codes, const uint8_t* a_sf, float ga,
+                         const uint8_t* b_codes, const uint8_t* b_sf, float gb,
+                         int64_t M, int64_t N, int64_t K,
+                         const int64_t* ii, const int64_t* jj, int64_t n,
+                         float* D, float* T);
+
+/* Scale-factor storage in 128-row x 4-block tiles of 512 bytes (the layout the
+ * Blackwell block-scaled MMA consumes): byte offset of scale (r, kb) for a
+ * tensor with n_kb blocks per row, total padded size, and a linear->tiled copy
+ * that zero-fills the padding. */
+int64_t nvfp4o_sf_swizzled_offset(int64_t r, int64_t kb, int64_t n_kb);
+int64_t nvfp4o_sf_swizzled_bytes(int64_t Rq, int64_t n_kb);
+void nvfp4o_sf_swizzle(const uint8_t* linear, int64_t Rq, int64_t n_kb, uint8_t* out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,418 @@
+"""Pins for the CPU oracle: each test fixes oracle behaviour with something other
+than the oracle itself -- the format definitions, exhaustive search in exact
+rational arithmetic, closed forms, published known-answer vectors, a library cast."""
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import binding as ob
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(name):
+    out = []
+    for line in open(os.path.join(GOLDEN, name)):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            out.append(line.split())
+    return out
+
+
+GRID = [float(v) for _, v in _rows("e2m1_grid.txt")]
+GRID_F = [Fraction(v) for v in GRID]
+# every E4M3 bit pattern decoded by the library cast (independent of the oracle)
+E4M3_LIB = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).float().numpy()
+
+
+# ---------------------------------------------------------------- formats
+def test_e2m1_decode_matches_grid():
+    for code in range(16):
+        mag = GRID[code & 7]
+        assert ob.e2m1_decode(code) == (-mag if code & 8 else mag)
+    # sign of zero is kept as a code but decodes to (-)0
+    assert np.signbit(np.float32(ob.e2m1_decode(8)))
+
+
+def test_e4m3_decode_matches_library_cast():
+    for code in range(127):
+        assert ob.e4m3_decode(code) == float(E4M3_LIB[code])
+    assert ob.e4m3_decode(0x7E) == 448.0
+    assert ob.e4m3_decode(1) == 2.0 ** -9
+    assert ob.e4m3_decode(8) == 2.0 ** -6
+
+
+def test_e4m3_roundtrip_all_finite_codes():
+    for code in range(127):
+        assert ob.e4m3_encode(ob.e4m3_decode(code)) == code
+
+
+def test_e4m3_encode_matches_library_cast_in_range():
+    rng = np.random.default_rng(0)
+    v = np.concatenate([
+        np.exp(rng.uniform(np.log(2.0 ** -12), np.log(448.0), 20000)),
+        rng.uniform(0, 2.0 ** -5, 2000), rng.uniform(400, 448, 500)]).astype(np.float32)
+    lib = torch.from_numpy(v).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    ours = np.array([ob.e4m3_encode(x) for x in v], dtype=np.uint8)
+    assert np.array_equal(lib, ours)
+
+
+def test_e4m3_encode_is_nearest_with_even_ties():
+    vals = [Fraction(float(E4M3_LIB[c])) for c in range(127)]
+    # exact midpoints between neighbours go to the even code
+    for c in range(126):
+        mid = (vals[c] + vals[c + 1]) / 2
+        got = ob.e4m3_encode(float(mid))
+        assert got == (c if c % 2 == 0 else c + 1), (c, float(mid), got)
+        # just off the midpoint goes to the nearer side
+        for eps, want in ((-1, c), (1, c + 1)):
+            x = np.nextafter(np.float32(float(mid)), np.float32(np.inf if eps > 0 else 0))
+            assert ob.e4m3_encode(float(x)) == want
+    # brute force: nearest in exact arithmetic
+    rng = np.random.default_rng(1)
+    for x in np.exp(rng.uniform(np.log(1e-4), np.log(447.0), 3000)).astype(np.float32):
+        fx = Fraction(float(x))
+        dist = [abs(fx - v) for v in vals]
+        best = min(dist)
+        got = ob.e4m3_encode(float(x))
+        assert dist[got] == best
+
+
+def test_e4m3_encode_saturates_and_handles_zero():
+    assert ob.e4m3_encode(0.0) == 0
+    assert ob.e4m3_encode(448.0) == 0x7E
+    assert ob.e4m3_encode(449.0) == 0x7E
+    assert ob.e4m3_encode(463.9) == 0x7E
+    assert ob.e4m3_encode(1e9) == 0x7E
+    assert ob.e4m3_encode(float("inf")) == 0x7E
+    assert ob.e4m3_encode(2.0 ** -10) == 0            # tie between 0 and the least subnormal
+    assert ob.e4m3_encode(float(np.nextafter(np.float32(2.0 ** -10), np.float32(1)))) == 1
+
+
+# ---------------------------------------------------------------- Philox
+def test_philox_known_answers():
+    for row in _rows("philox4x32_10_kat.txt"):
+        v = [int(t, 16) for t in row]
+        out = ob.philox4x32_10(v[4:6], v[0:4])
+        assert [int(o) for o in out] == v[6:10]
+
+
+def test_block_random_bytes_are_little_endian_words_of_the_counter():
+    seed, offset, block = 0x0123456789ABCDEF, 0x1122334455667788, 0xA1B2C3D4E5F60718
+    words = ob.philox4x32_10([seed & 0xFFFFFFFF, seed >> 32],
+                             [block & 0xFFFFFFFF, block >> 32, offset & 0xFFFFFFFF, offset >> 32])
+    want = np.frombuffer(words.astype("<u4").tobytes(), dtype=np.uint8)
+    assert np.array_equal(ob.block_random_bytes(seed, offset, block), want)
+    # different block / offset / seed -> different bytes
+    assert not np.array_equal(ob.block_random_bytes(seed, offset, block + 1), want)
+    assert not np.array_equal(ob.block_random_bytes(seed, offset + 1, block), want)
+    assert not np.array_equal(ob.block_random_bytes(seed + 1, offset, block), want)
+
+
+# ---------------------------------------------------------------- rounding
+def test_rtn_golden_ties():
+    for y, code, val in _rows("rtn_ties.txt"):
+        assert ob.round_rtn(float(y)) == int(code)
+        assert GRID[int(code)] == float(val)
+
+
+def test_rtn_is_argmin_for_every_bf16_value_in_range():
+    # all non-negative bf16 bit patterns up to 6.0
+    bits = np.arange(0, 0x40C1, dtype=np.uint32)           # 0x40C0 = 6.0 in bf16
+    ys = (bits << 16).view(np.float32)
+    for y in ys:
+        fy = Fraction(float(y))
+        dist = [abs(fy - g) for g in GRID_F]
+        best = min(dist)
+        got = ob.round_rtn(float(y))
+        assert dist[got] == best
+        ties = [c for c in range(8) if dist[c] == best]
+        if len(ties) == 2:
+            assert got % 2 == 0
+
+
+def _sr_neighbours(y):
+    lo = max(g for g in GRID if g <= y)
+    hi = min(g for g in GRID if g >= y)
+    return lo, hi
+
+
+def test_sr_exact_distribution_over_all_bytes():
+    rng = np.random.default_rng(2)
+    ys = np.concatenate([rng.uniform(0, 6, 300), np.array(GRID), [0.001, 5.999, 1.999, 2.001, 3.999, 4.001]])
+    for y in ys.astype(np.float32):
+        lo, hi = _sr_neighbours(float(y))
+        vals = np.array([GRID[ob.round_sr(float(y), u)] for u in range(256)])
+        assert set(vals.tolist()) <= {lo, hi}
+        if lo == hi:                                         # representable values never move
+            assert np.all(vals == lo)
+            continue
+        delta = hi - lo
+        f = (Fraction(float(y)) - Fraction(lo)) / Fraction(delta)
+        ups = sum(1 for u in range(256) if Fraction(2 * u + 1, 512) < f)
+        assert int(np.sum(vals == hi)) == ups
+        # rounding up happens for the smallest bytes (monotone in u)
+        assert np.all(np.diff((vals == hi).astype(int)) <= 0)
+        assert abs(vals.mean() - float(y)) <= delta / 512 + 1e-12
+
+
+def test_sr_unbiased_over_seeded_draws():
+    # 10^4 Philox-seeded draws of the same block: mean within 3 sigma (+ the 8-bit bias bound)
+    x = np.array([[0.3, -0.7, 1.1, 1.6, 2.2, -2.9, 3.3, 4.7, 5.5, 0.05, 6.0, -0.26, 0.9, 1.9, 3.9, -5.9]],
+                 dtype=np.float32)
+    n = 10000
+    acc = np.zeros(16)
+    acc2 = np.zeros(16)
+    for s in range(n):
+        codes, scales = ob.quantize(x, mode=ob.SR, seed=s, offset=7, nthreads=1)
+        assert scales[0, 0] == ob.e4m3_encode(1.0)           # amax 6 -> scale 1
+        deq = ob.dequantize(codes, scales)[0].astype(np.float64)
+        acc += deq
+        acc2 += deq * deq
+    mean = acc / n
+    var = np.maximum(acc2 / n - mean ** 2, 0)
+    for j in range(16):
+        lo, hi = _sr_neighbours(abs(float(x[0, j])))
+        bound = 3 * np.sqrt(var[j] / n) + (hi - lo) / 512 + 1e-9
+        assert abs(mean[j] - float(x[0, j])) <= bound, (j, mean[j], x[0, j], bound)
+
+
+def test_sr_variance_closed_form():
+    # y uniform within one grid step: E[err^2] = delta^2/6 under SR, delta^2/12 under RtN
+    rng = np.random.default_rng(3)
+    ys = rng.uniform(2.0, 3.0, 40000).astype(np.float32)
+    us = rng.integers(0, 256, ys.size)
+    sr = np.array([GRID[ob.round_sr(float(y), int(u))] for y, u in zip(ys, us)])
+    rt = np.array([GRID[ob.round_rtn(float(y))] for y in ys])
+    assert abs(np.mean((sr - ys) ** 2) - 1 / 6) < 0.01
+    assert abs(np.mean((rt - ys) ** 2) - 1 / 12) < 0.005
+    assert abs(np.mean(sr - ys)) < 0.01
+
+
+# ---------------------------------------------------------------- block quantizer
+def _exact_block_check(x, codes, scales):
+    """Exhaustive-search definition in rational arithmetic: the scale is a nearest
+    E4M3 value to amax/6 and every code a nearest grid value to |x|/scale (up to
+    the fp32 roundings the oracle is allowed: a relative slack of 2^-20)."""
+    e4 = [Fraction(float(E4M3_LIB[c])) for c in range(127)]
+    R, K = x.shape
+    for r in range(R):
+        for kb in range(K // 16):
+            blk = x[r, kb * 16:(kb + 1) * 16]
+            amax = Fraction(float(np.max(np.abs(blk))))
+            target = amax / 6
+            dist = [abs(target - v) for v in e4]
+            sq = int(scales[r, kb])
+            assert dist[sq] <= min(dist) + target * Fraction(1, 2 ** 20)
+            s = e4[sq]
+            for j in range(16):
+                byte = codes[r, (kb * 16 + j) // 2]
+                nib = (byte >> 4) if j & 1 else (byte & 15)
+                assert (nib >> 3) == int(np.signbit(blk[j]))
+                if s == 0:
+                    assert nib & 7 == 0
+                    continue
+                y = min(abs(Fraction(float(blk[j]))) / s, Fraction(6))
+                d = [abs(y - g) for g in GRID_F]
+                assert d[nib & 7] <= min(d) + y * Fraction(1, 2 ** 20)
+
+
+def test_quantize_rtn_brute_force_tiny():
+    rng = np.random.default_rng(4)
+    for scale in (1.0, 0.02, 37.0):
+        x = (rng.standard_normal((3, 48)) * scale).astype(np.float32)
+        x = torch.from_numpy(x).to(torch.bfloat16).float().numpy()
+        codes, scales = ob.quantize(x, nthreads=1)
+        _exact_block_check(x, codes, scales)
+
+
+def test_quantize_layout_nibbles_and_scale_index():
+    # one non-zero element at a time: its nibble position and block scale index are fixed
+    for (r, k) in [(0, 0), (0, 1), (1, 17), (2, 46), (1, 31)]:
+        x = np.zeros((3, 48), dtype=np.float32)
+        x[r, k] = -3.0                                      # amax 3 -> scale 0.5, value 6 -> code 7, sign 1
+        codes, scales = ob.quantize(x, nthreads=1)
+        want_codes = np.zeros_like(codes)
+        want_codes[r, k // 2] = 0xF << (4 * (k & 1))
+        want_scales = np.zeros_like(scales)
+        want_scales[r, k // 16] = ob.e4m3_encode(0.5)
+        assert np.array_equal(codes, want_codes)
+        assert np.array_equal(scales, want_scales)
+        assert ob.e4m3_decode(int(scales[r, k // 16])) == 0.5
+
+
+def test_quantize_scale_invariants():
+    rng = np.random.default_rng(5)
+    x = torch.from_numpy(rng.standard_normal((8, 256)).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    codes, scales = ob.quantize(x, nthreads=1)
+    # amax maps near 6: the largest magnitude code of every normal-scale block is 7
+    mags = np.maximum(codes & 7, (codes >> 4) & 7).reshape(8, 16, 8).max(axis=2)
+    assert np.all(mags[scales >= 8] == 7)
+    # power-of-two equivariance: same codes, scale exponent shifted
+    for k in (-3, 2):
+        c2, s2 = ob.quantize(x * np.float32(2.0 ** k), nthreads=1)
+        assert np.array_equal(c2, codes)
+        assert np.array_equal(s2.astype(int), scales.astype(int) + 8 * k)
+    # idempotence under RtN
+    deq = ob.dequantize(codes, scales)
+    c3, s3 = ob.quantize(deq, nthreads=1)
+    assert np.array_equal(c3, codes) and np.array_equal(s3, scales)
+    # sign symmetry
+    c4, s4 = ob.quantize(-x, nthreads=1)
+    assert np.array_equal(c4, codes ^ 0x88) and np.array_equal(s4, scales)
+
+
+def test_quantize_zero_block_and_underflow():
+    x = np.zeros((1, 32), dtype=np.float32)
+    x[0, 3] = -0.0
+    x[0, 16:] = 1e-4                                         # amax/6 far below the smallest E4M3 step
+    codes, scales = ob.quantize(x, nthreads=1)
+    assert np.all(scales == 0)
+    want = np.zeros((1, 16), dtype=np.uint8)
+    want[0, 1] = 0x80                                        # only the sign bit of -0.0 survives
+    assert np.array_equal(codes, want)
+    assert np.all(np.isfinite(ob.dequantize(codes, scales)))
+
+
+def test_quantize_saturating_scale_clamps_values():
+    x = np.full((1, 16), 10.0, dtype=np.float32)
+    x[0, 0] = 6.0 * 448.0 * 4                                # scale saturates at 448, value/scale = 24 -> clamp 6
+    codes, scales = ob.quantize(x, nthreads=1)
+    assert scales[0, 0] == 0x7E
+    assert codes[0, 0] & 7 == 7
+
+
+def test_quantize_global_scale():
+    rng = np.random.default_rng(6)
+    x = torch.from_numpy((rng.standard_normal((4, 64)) * 1e-4).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    g = ob.tensor_amax_scale(x)
+    assert g == float(np.float32(np.max(np.abs(x))) / np.float32(2688.0))
+    codes, scales = ob.quantize(x, g=g, nthreads=1)
+    assert scales.max() == 0x7E or scales.max() == 0x7D      # the largest block lands at (or next to) 448
+    # with a power-of-two g the result equals quantizing x/g without g
+    g2 = 2.0 ** -20
+    c1, s1 = ob.quantize(x, g=g2, nthreads=1)
+    c2, s2 = ob.quantize(x / np.float32(g2), nthreads=1)
+    assert np.array_equal(c1, c2) and np.array_equal(s1, s2)
+    deq = ob.dequantize(c1, s1, g=g2)
+    assert np.max(np.abs(deq - x)) <= np.max(np.abs(x)) * 0.26
+    assert ob.tensor_amax_scale(np.zeros(5, dtype=np.float32)) == 1.0
+
+
+def test_quantize_sr_uses_block_indexed_bytes_and_is_reproducible():
+    rng = np.random.default_rng(7)
+    x = torch.from_numpy(rng.standard_normal((5, 64)).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    c1, s1 = ob.quantize(x, mode=ob.SR, seed=11, offset=3, nthreads=1)
+    c2, s2 = ob.quantize(x, mode=ob.SR, seed=11, offset=3, nthreads=4)
+    assert np.array_equal(c1, c2) and np.array_equal(s1, s2)
+    c3, _ = ob.quantize(x, mode=ob.SR, seed=11, offset=4, nthreads=1)
+    assert not np.array_equal(c1, c3)
+    crt, srt = ob.quantize(x, nthreads=1)
+    assert np.array_equal(srt, s1)                           # scales do not depend on the rounding mode
+    # rebuild every code from the per-element rule and the bytes of block r*(K/16)+kb
+    for r in range(5):
+        for kb in range(4):
+            rnd = ob.block_random_bytes(11, 3, r * 4 + kb)
+            d = np.float32(ob.e4m3_decode(int(s1[r, kb])))
+            inv = np.float32(1.0) / d
+            for j in range(16):
+                v = x[r, kb * 16 + j]
+                y = min(np.float32(abs(v)) * inv, np.float32(6.0))
+                m = ob.round_sr(float(y), int(rnd[j]))
+                byte = c1[r, (kb * 16 + j) // 2]
+                nib = (byte >> 4) if j & 1 else (byte & 15)
+                assert nib == (m | (8 if np.signbit(v) else 0))
+
+
+def test_quantize_transposed_is_row_quantize_of_the_transpose():
+    rng = np.random.default_rng(8)
+    x = torch.from_numpy(rng.standard_normal((32, 24)).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    for mode in (ob.RTN, ob.SR):
+        ct, st = ob.quantize(x, mode=mode, seed=5, offset=1, transposed=True, nthreads=1)
+        cr, sr_ = ob.quantize(np.ascontiguousarray(x.T), mode=mode, seed=5, offset=1, nthreads=1)
+        assert ct.shape == (24, 16) and st.shape == (24, 2)
+        assert np.array_equal(ct, cr) and np.array_equal(st, sr_)
+
+
+# ---------------------------------------------------------------- scale layout
+def test_swizzled_scale_layout_structure():
+    for Rq, nkb in [(128, 4), (256, 8), (130, 5), (1, 1), (384, 12)]:
+        total = ob.sf_swizzled_bytes(Rq, nkb)
+        assert total == -(-Rq // 128) * -(-nkb // 4) * 512
+        offs = np.array([[ob.sf_swizzled_offset(r, kb, nkb) for kb in range(nkb)] for r in range(Rq)])
+        assert len(np.unique(offs)) == Rq * nkb and offs.min() >= 0 and offs.max() < total
+        if Rq % 128 == 0 and nkb % 4 == 0:
+            assert sorted(offs.reshape(-1).tolist()) == list(range(total))   # a permutation
+        lin = np.arange(Rq * nkb, dtype=np.uint32).astype(np.uint8).reshape(Rq, nkb)
+        sw = ob.sf_swizzle(lin)
+        assert np.array_equal(sw[offs.reshape(-1)], lin.reshape(-1))
+        mask = np.ones(total, bool)
+        mask[offs.reshape(-1)] = False
+        assert np.all(sw[mask] == 0)
+    o = lambda r, kb: ob.sf_swizzled_offset(r, kb, 8)
+    # one 128x4 tile is 512 contiguous bytes; 4 blocks of a row are adjacent; rows r, r+32,
+    # r+64, r+96 share a 16-byte group; consecutive rows are 16 bytes apart
+    assert o(0, 0) == 0 and o(0, 3) == 3 and o(0, 4) == 512 and o(128, 0) == 1024
+    assert o(1, 0) == 16 and o(31, 0) == 31 * 16
+    assert o(32, 0) == 4 and o(64, 0) == 8 and o(96, 0) == 12 and o(127, 3) == 511
+
+
+# ---------------------------------------------------------------- GEMM
+def _rand_quantized(rng, R, K, std=1.0):
+    x = torch.from_numpy((rng.standard_normal((R, K)) * std).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    return ob.quantize(x, nthreads=1)
+
+
+def test_gemm_matches_library_matmul_in_float64():
+    rng = np.random.default_rng(9)
+    ac, asf = _rand_quantized(rng, 7, 96)
+    bc, bsf = _rand_quantized(rng, 5, 96, std=0.02)
+    ga, gb = 0.5, 2.0 ** -3
+    D, T = ob.gemm(ac, asf, ga, bc, bsf, gb)
+    A = torch.from_numpy(ob.dequantize(ac, asf)).double() * ga
+    B = torch.from_numpy(ob.dequantize(bc, bsf)).double() * gb
+    ref = (A @ B.T).numpy()
+    refT = (A.abs() @ B.abs().T).numpy()
+    assert np.allclose(D, ref, rtol=1e-6, atol=0)
+    assert np.allclose(T, refT, rtol=1e-6, atol=0)
+    Ds, Ts = ob.gemm_sampled(ac, asf, ga, bc, bsf, gb, [0, 6, 3], [4, 0, 2])
+    assert np.array_equal(Ds, D[[0, 6, 3], [4, 0, 2]]) and np.array_equal(Ts, T[[0, 6, 3], [4, 0, 2]])
+    D32 = ob.gemm_f32acc(ac, asf, ga, bc, bsf, gb)
+    assert np.all(np.abs(D32 - D) <= 1e-6 * T)
+
+
+def test_gemm_exact_small_integers_and_one_hot():
+    # power-of-two scales, small K: every partial sum is exact -> equality with integer arithmetic
+    rng = np.random.default_rng(10)
+    grid = np.array(GRID + [-g for g in GRID], dtype=np.float32)
+    A = rng.choice(grid, size=(6, 32))
+    A[:, 0] = 6.0
+    A[:, 16] = -6.0                                          # amax 6 per block -> scale exactly 1
+    B = rng.choice(grid, size=(4, 32))
+    B[:, 1] = 6.0
+    B[:, 17] = 6.0
+    ac, asf = ob.quantize(A.astype(np.float32), nthreads=1)
+    bc, bsf = ob.quantize(B.astype(np.float32), nthreads=1)
+    assert np.all(asf == ob.e4m3_encode(1.0)) and np.all(bsf == ob.e4m3_encode(1.0))
+    D, T = ob.gemm(ac, asf, 1.0, bc, bsf, 1.0)
+    assert np.array_equal(D, (A.astype(np.float64) @ B.astype(np.float64).T).astype(np.float32))
+    # a one-hot row of A reads back a column of dequantized B
+    E = np.zeros((32, 32), dtype=np.float32)
+    E[np.arange(32), np.arange(32)] = 6.0
+    ec, esf = ob.quantize(E, nthreads=1)
+    D2 = ob.gemm(ec, esf, 1.0, bc, bsf, 1.0, want_T=False)
+    assert np.array_equal(D2, 6.0 * ob.dequantize(bc, bsf).T)
+
+
+def test_gemm_transposed_operand_detected():
+    # a swapped-operand or transposed-output mistake changes the shape-asymmetric result
+    rng = np.random.default_rng(11)
+    ac, asf = _rand_quantized(rng, 3, 32)
+    bc, bsf = _rand_quantized(rng, 5, 32)
+    D = ob.gemm(ac, asf, 1.0, bc, bsf, 1.0, want_T=False)
+    A, B = ob.dequantize(ac, asf).astype(np.float64), ob.dequantize(bc, bsf).astype(np.float64)
+    assert D.shape == (3, 5)
+    assert np.allclose(D, A @ B.T, rtol=1e-6)
