@@ -1,0 +1,168 @@
+/*
+ * nvfp4.h -- C ABI of the B200 (sm_100a) NVFP4 quantize-then-GEMM library.
+ *
+ * The library implements the quantized linear layer of "FP4 All the Way: Fully
+ * Quantized Training of LLMs": every operand of the three training GEMMs
+ * (Eq. 1-3) is cut into blocks of 16 values along the contraction axis, each
+ * block gets an E4M3 scale, and values become 4-bit E2M1 codes (Section 3),
+ * rounded to nearest in the forward pass and stochastically in the backward and
+ * update passes (Eq. 4-6).
+ *
+ * Conventions for every entry point
+ *   - Returns an nvfp4_status (int).  Never throws, never exits the process.
+ *   - Pointers are DEVICE pointers unless the comment says "host".  The caller
+ *     owns every buffer; the library allocates no device memory (scratch comes
+ *     from the caller's workspace).
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL =
+ *     the legacy default stream) and is asynchronous; there is no internal
+ *     synchronisation.  Argument errors are detected on the host before any
+ *     launch; launch failures map to NVFP4_ERR_CUDA.
+ *   - Tensors are row-major.  M = tokens, K = in-features, N = out-features.
+ *   - Packed codes: element 2i sits in bits 0-3 and element 2i+1 in bits 4-7 of
+ *     byte i.  A code is sign<<3 | exponent(2)<<1 | mantissa(1).
+ *   - "Quantized shape" (Rq, Kq): for transposed == 0 it is (rows, cols); for
+ *     transposed == 1 it is (cols, rows).  Blocks always run along Kq, codes are
+ *     stored [Rq, Kq/2] and scales [Rq, Kq/16], so Kq is the contiguous
+ *     (contraction) axis of the output.  Kq must be a multiple of 16.
+ */
+#ifndef NVFP4_H
+#define NVFP4_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define NVFP4_API __attribute__((visibility("default")))
+#else
+#define NVFP4_API
+#endif
+
+typedef enum {
+  NVFP4_OK = 0,
+  NVFP4_ERR_NULL = 1,       /* a required pointer is NULL */
+  NVFP4_ERR_SHAPE = 2,      /* non-positive size, contraction length not a multiple of 16, ld too small */
+  NVFP4_ERR_ALIGN = 3,      /* a base pointer or leading dimension breaks the alignment rule below */
+  NVFP4_ERR_ENUM = 4,       /* unknown dtype / rounding mode / layout / flag */
+  NVFP4_ERR_WORKSPACE = 5,  /* workspace missing or smaller than nvfp4_linear_workspace_bytes */
+  NVFP4_ERR_ARCH = 6,       /* current device is not compute capability 10.x */
+  NVFP4_ERR_CUDA = 7        /* a CUDA runtime/driver call or a launch failed */
+} nvfp4_status;
+
+typedef enum { NVFP4_BF16 = 0, NVFP4_FP32 = 1 } nvfp4_dtype;
+typedef enum { NVFP4_RTN = 0, NVFP4_SR = 1 } nvfp4_round_mode;
+typedef enum { NVFP4_SF_LINEAR = 0, NVFP4_SF_SWIZZLED_128x4 = 1 } nvfp4_sf_layout;
+typedef enum { NVFP4_G_NONE = 0, NVFP4_G_AMAX = 1, NVFP4_G_GIVEN = 2 } nvfp4_gscale_mode;
+typedef enum { NVFP4_LINEAR_FWD = 0, NVFP4_LINEAR_BWD_DX = 1, NVFP4_LINEAR_BWD_DW = 2 } nvfp4_linear_kind;
+
+/* Rounding of one operand, chosen per call (Eq. 4-6 fix the paper's choice per
+ * site; any site may be overridden, as the paper's per-site ablation does).
+ * For NVFP4_SR the random byte of element j of block B (B = r*(Kq/16) + kb in
+ * the quantized shape) is byte j of Philox4x32-10 with key = seed and counter =
+ * (B, offset); the same (seed, offset) reproduces the same codes. */
+typedef struct {
+  int32_t mode;      /* nvfp4_round_mode */
+  int32_t reserved;  /* must be 0 */
+  uint64_t seed;
+  uint64_t offset;
+} nvfp4_rounding;
+
+/* Text for a status code (host pointer to a static string). */
+NVFP4_API const char* nvfp4_status_string(int status);
+
+/* Bytes of a scale buffer for a quantized shape (Rq, Kq): linear = Rq*Kq/16;
+ * swizzled = ceil(Rq/128)*ceil(Kq/64)*512.  Returns 0 on bad arguments. */
+NVFP4_API size_t nvfp4_sf_bytes(int64_t Rq, int64_t Kq, int sf_layout);
+
+/*
+ * Quantizer Q(x) of Section 3 / Eq. 4-6: per block of 16 along Kq,
+ *   scale  = E4M3( amax * ((1/6)/g) )   nearest-even, saturating at 448, sign unused
+ *   code_j = E2M1( min(|x_j| / (decode(scale)*g), 6) )   RtN (ties to even) or SR,
+ * sign kept.  g is *global_scale (NULL => 1.0f), a per-tensor fp32 factor.
+ *
+ *   x            [rows, cols] of `dtype`, leading dimension ld (elements, >= cols)
+ *   transposed   0: blocks along cols.  1: blocks along rows and the output is
+ *                stored transposed (quantized shape (cols, rows))
+ *   codes        Rq*Kq/2 bytes;  scales  nvfp4_sf_bytes(Rq, Kq, sf_layout) bytes.
+ *                In the swizzled layout scale (r, kb) lives at
+ *                ((r/128)*ceil(Kq/64) + kb/4)*512 + (r%32)*16 + ((r%128)/32)*4 + kb%4
+ *                and padding bytes are written as 0.
+ * Alignment: x, codes, scales 16-byte aligned; ld a multiple of 8 elements.
+ * Errors: NULL pointers, Kq % 16 != 0, ld < cols, bad enums, misalignment.
+ */
+NVFP4_API int nvfp4_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                   int transposed, const float* global_scale, const nvfp4_rounding* rounding /* host */,
+                   uint8_t* codes, uint8_t* scales, int sf_layout, void* cuda_stream);
+
+/* Per-tensor scale g = max|x| / (6*448), or 1.0f for an all-zero tensor, written
+ * to *global_scale_out (device).  The paper defines only the block scale; this
+ * optional factor keeps small-magnitude gradients inside the E4M3 scale range. */
+NVFP4_API int nvfp4_tensor_amax_scale(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                            float* global_scale_out, void* cuda_stream);
+
+/*
+ * Block-scaled GEMM (the contraction of Eq. 1-3 on quantized operands):
+ *   D[m,n] = (gA*gB) * sum_kb sA[m,kb]*sB[n,kb] * sum_{k in kb} a[m,k]*b[n,k]
+ * A is [M,K] and B is [N,K], both K-major packed codes with scales in the
+ * swizzled layout; a_g / b_g are device fp32 per-tensor scales (NULL => 1).
+ * D is [M,N] row-major, leading dimension ldd (elements), fp32 or bf16;
+ * accumulation is fp32.  K % 16 == 0; code rows are K/2 bytes (so K % 32 == 0
+ * is required for the 16-byte row pitch of the tiled copies); ldd*sizeof(D)
+ * a multiple of 16; all base pointers 16-byte aligned.
+ */
+NVFP4_API int nvfp4_gemm(const uint8_t* a_codes, const uint8_t* a_sf, const float* a_g,
+               const uint8_t* b_codes, const uint8_t* b_sf, const float* b_g,
+               int64_t M, int64_t N, int64_t K,
+               void* d, int d_dtype, int64_t ldd, void* cuda_stream);
+
+/* Tuning/testing hook: force the GEMM tile width (128 or 256 output columns per
+ * CTA tile); 0 restores the automatic choice.  Process-wide, not thread-safe. */
+NVFP4_API int nvfp4_gemm_set_tile_n(int bn);
+
+/* Scratch bytes nvfp4_linear_* needs for a layer of shape (M, N, K);
+ * `which` is an nvfp4_linear_kind.  Returns 0 on bad arguments. */
+NVFP4_API size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int which);
+
+/*
+ * Forward pass, Eq. 1 / Eq. 4:  Y[M,N] = Q(X)[M,K] . Q(W)[N,K]^T, blocks along K.
+ * rx / rw (host) choose the rounding (the paper: RtN for both).
+ * gscale_mode: NVFP4_G_NONE  g = 1 for both operands;
+ *              NVFP4_G_AMAX  g computed here from each operand's amax (one extra read);
+ *              NVFP4_G_GIVEN gx / gw are device pointers supplied by the caller.
+ * X, W of `dtype` (dense, ld = K); Y of y_dtype (dense, ld = N).
+ * workspace: device scratch of at least nvfp4_linear_workspace_bytes(M,N,K,FWD),
+ * 256-byte aligned; its contents are undefined afterwards.
+ */
+NVFP4_API int nvfp4_linear_fwd(const void* X, const void* W, int dtype, int64_t M, int64_t N, int64_t K,
+                     int gscale_mode, const float* gx, const float* gw,
+                     const nvfp4_rounding* rx, const nvfp4_rounding* rw,
+                     void* Y, int y_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Backward pass, Eq. 2 / Eq. 5:  dX[M,K] = Q(dY)[M,N] . Q(W^T)[K,N]^T, blocks
+ * along N: dY is quantized along its rows' contiguous axis, W is quantized
+ * transposed.  The paper: SR for dY, RtN for W^T. */
+NVFP4_API int nvfp4_linear_bwd_dx(const void* dY, const void* W, int dtype, int64_t M, int64_t N, int64_t K,
+                        int gscale_mode, const float* gdy, const float* gw,
+                        const nvfp4_rounding* rdy, const nvfp4_rounding* rw,
+                        void* dX, int dx_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Update pass (weight gradient), Eq. 3 / Eq. 6:  dW[N,K] = Q(dY^T)[N,M] . Q(X^T)[K,M]^T,
+ * blocks along the token axis M: both operands are quantized transposed.
+ * The paper: SR for both. */
+NVFP4_API int nvfp4_linear_bwd_dw(const void* dY, const void* X, int dtype, int64_t M, int64_t N, int64_t K,
+                        int gscale_mode, const float* gdy, const float* gx,
+                        const nvfp4_rounding* rdy, const nvfp4_rounding* rx,
+                        void* dW, int dw_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Reads and clears the device-side error word of the current device (host
+ * out-pointer; synchronises the device).  Non-zero means a kernel gave up on a
+ * bounded wait and its output is invalid; bits 0-7 identify the wait site. */
+NVFP4_API int nvfp4_device_error_word(uint32_t* host_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

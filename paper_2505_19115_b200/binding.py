@@ -1,0 +1,197 @@
+"""Thin ctypes binding over libnvfp4.so: argument marshalling only.
+
+Every function has the name of the C entry point it calls (include/nvfp4.h).
+torch tensors are used for device memory and streams; all computation happens
+inside the CUDA library.  There is no CPU fallback: if the library is missing
+or a call fails, an exception is raised.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnvfp4.so")
+
+BF16, FP32 = 0, 1
+RTN, SR = 0, 1
+SF_LINEAR, SF_SWIZZLED = 0, 1
+G_NONE, G_AMAX, G_GIVEN = 0, 1, 2
+LINEAR_FWD, LINEAR_BWD_DX, LINEAR_BWD_DW = 0, 1, 2
+
+
+class NvFp4Error(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: nvfp4 status {status} ({status_string(status)})")
+
+
+class Rounding(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("reserved", C.c_int32), ("seed", C.c_uint64), ("offset", C.c_uint64)]
+
+    def __init__(self, mode=RTN, seed=0, offset=0):
+        super().__init__(mode, 0, seed, offset)
+
+
+_lib = None
+
+
+def lib():
+    """Load libnvfp4.so (built in-tree by paper_2505_19115_b200/build.py).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} not found: build it with `python -m paper_2505_19115_b200.build` "
+                           "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i64, ci, sz = C.c_void_p, C.c_int64, C.c_int, C.c_size_t
+    rp = C.POINTER(Rounding)
+    L.nvfp4_status_string.restype = C.c_char_p
+    L.nvfp4_status_string.argtypes = [ci]
+    L.nvfp4_sf_bytes.restype = sz
+    L.nvfp4_sf_bytes.argtypes = [i64, i64, ci]
+    L.nvfp4_quantize.restype = ci
+    L.nvfp4_quantize.argtypes = [vp, ci, i64, i64, i64, ci, vp, rp, vp, vp, ci, vp]
+    L.nvfp4_tensor_amax_scale.restype = ci
+    L.nvfp4_tensor_amax_scale.argtypes = [vp, ci, i64, i64, i64, vp, vp]
+    L.nvfp4_gemm.restype = ci
+    L.nvfp4_gemm.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, i64, vp]
+    L.nvfp4_gemm_set_tile_n.restype = ci
+    L.nvfp4_gemm_set_tile_n.argtypes = [ci]
+    L.nvfp4_linear_workspace_bytes.restype = sz
+    L.nvfp4_linear_workspace_bytes.argtypes = [i64, i64, i64, ci]
+    lin = [vp, vp, ci, i64, i64, i64, ci, vp, vp, rp, rp, vp, ci, vp, sz, vp]
+    for name in ("nvfp4_linear_fwd", "nvfp4_linear_bwd_dx", "nvfp4_linear_bwd_dw"):
+        getattr(L, name).restype = ci
+        getattr(L, name).argtypes = lin
+    L.nvfp4_device_error_word.restype = ci
+    L.nvfp4_device_error_word.argtypes = [C.POINTER(C.c_uint32)]
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().nvfp4_status_string(status).decode()
+
+
+def _check(status, where):
+    if status != 0:
+        raise NvFp4Error(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return FP32
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def nvfp4_sf_bytes(Rq: int, Kq: int, sf_layout: int = SF_SWIZZLED) -> int:
+    return int(lib().nvfp4_sf_bytes(Rq, Kq, sf_layout))
+
+
+def nvfp4_quantize(x: torch.Tensor, transposed: bool = False, global_scale: torch.Tensor = None,
+                   rounding: Rounding = None, sf_layout: int = SF_LINEAR, codes: torch.Tensor = None,
+                   scales: torch.Tensor = None, stream=None):
+    """Returns (codes [Rq, Kq/2] u8, scales u8: [Rq, Kq/16] linear or a flat swizzled buffer)."""
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    Rq, Kq = (cols, rows) if transposed else (rows, cols)
+    rounding = rounding or Rounding()
+    if codes is None:
+        codes = torch.empty((Rq, max(Kq // 2, 1)), dtype=torch.uint8, device=x.device)
+    if scales is None:
+        if sf_layout == SF_LINEAR:
+            scales = torch.empty((Rq, max(Kq // 16, 1)), dtype=torch.uint8, device=x.device)
+        else:
+            scales = torch.empty(max(nvfp4_sf_bytes(Rq, Kq, sf_layout), 16), dtype=torch.uint8, device=x.device)
+    st = lib().nvfp4_quantize(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), int(transposed),
+                              _ptr(global_scale), C.byref(rounding), _ptr(codes), _ptr(scales), sf_layout,
+                              _stream(stream))
+    _check(st, "nvfp4_quantize")
+    return codes, scales
+
+
+def nvfp4_tensor_amax_scale(x: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+    if out is None:
+        out = torch.empty(1, dtype=torch.float32, device=x.device)
+    st = lib().nvfp4_tensor_amax_scale(_ptr(x), _dtype_code(x), x.shape[0], x.shape[1], x.stride(0), _ptr(out),
+                                       _stream(stream))
+    _check(st, "nvfp4_tensor_amax_scale")
+    return out
+
+
+def nvfp4_gemm(a_codes, a_sf, a_g, b_codes, b_sf, b_g, out_dtype=torch.float32, out: torch.Tensor = None,
+               stream=None) -> torch.Tensor:
+    """D[M,N] = A[M,K] . B[N,K]^T on packed codes with swizzled scales."""
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    N = b_codes.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=a_codes.device)
+    st = lib().nvfp4_gemm(_ptr(a_codes), _ptr(a_sf), _ptr(a_g), _ptr(b_codes), _ptr(b_sf), _ptr(b_g),
+                          M, N, K, _ptr(out), _dtype_code(out), out.stride(0), _stream(stream))
+    _check(st, "nvfp4_gemm")
+    return out
+
+
+def nvfp4_gemm_set_tile_n(bn: int) -> None:
+    _check(lib().nvfp4_gemm_set_tile_n(bn), "nvfp4_gemm_set_tile_n")
+
+
+def nvfp4_linear_workspace_bytes(M: int, N: int, K: int, which: int) -> int:
+    return int(lib().nvfp4_linear_workspace_bytes(M, N, K, which))
+
+
+def _linear(name, which, a, b, M, N, K, out_shape, gscale_mode, ga, gb, ra, rb, out, out_dtype, workspace, stream):
+    if out is None:
+        out = torch.empty(out_shape, dtype=out_dtype, device=a.device)
+    if workspace is None:
+        workspace = torch.empty(nvfp4_linear_workspace_bytes(M, N, K, which), dtype=torch.uint8, device=a.device)
+    assert a.is_contiguous() and b.is_contiguous() and out.is_contiguous() and a.dtype == b.dtype
+    st = getattr(lib(), name)(_ptr(a), _ptr(b), _dtype_code(a), M, N, K, gscale_mode, _ptr(ga), _ptr(gb),
+                              C.byref(ra), C.byref(rb), _ptr(out), _dtype_code(out), _ptr(workspace),
+                              workspace.numel(), _stream(stream))
+    _check(st, name)
+    return out
+
+
+def nvfp4_linear_fwd(X, W, gscale_mode=G_AMAX, gx=None, gw=None, rx=None, rw=None, out=None,
+                     out_dtype=torch.float32, workspace=None, stream=None):
+    """Y[M,N] = Q(X) . Q(W)^T (Eq. 1/4).  Default rounding: RtN for both."""
+    (M, K), N = X.shape, W.shape[0]
+    return _linear("nvfp4_linear_fwd", LINEAR_FWD, X, W, M, N, K, (M, N), gscale_mode, gx, gw,
+                   rx or Rounding(RTN), rw or Rounding(RTN), out, out_dtype, workspace, stream)
+
+
+def nvfp4_linear_bwd_dx(dY, W, gscale_mode=G_AMAX, gdy=None, gw=None, rdy=None, rw=None, out=None,
+                        out_dtype=torch.float32, workspace=None, stream=None):
+    """dX[M,K] = Q(dY) . Q(W^T)^T (Eq. 2/5).  Default rounding: SR for dY, RtN for W^T."""
+    (M, N), K = dY.shape, W.shape[1]
+    return _linear("nvfp4_linear_bwd_dx", LINEAR_BWD_DX, dY, W, M, N, K, (M, K), gscale_mode, gdy, gw,
+                   rdy or Rounding(SR, 0, 0), rw or Rounding(RTN), out, out_dtype, workspace, stream)
+
+
+def nvfp4_linear_bwd_dw(dY, X, gscale_mode=G_AMAX, gdy=None, gx=None, rdy=None, rx=None, out=None,
+                        out_dtype=torch.float32, workspace=None, stream=None):
+    """dW[N,K] = Q(dY^T) . Q(X^T)^T (Eq. 3/6).  Default rounding: SR for both."""
+    (M, N), K = dY.shape, X.shape[1]
+    return _linear("nvfp4_linear_bwd_dw", LINEAR_BWD_DW, dY, X, M, N, K, (N, K), gscale_mode, gdy, gx,
+                   rdy or Rounding(SR, 0, 1), rx or Rounding(SR, 0, 2), out, out_dtype, workspace, stream)
+
+
+def nvfp4_device_error_word() -> int:
+    w = C.c_uint32(0)
+    _check(lib().nvfp4_device_error_word(C.byref(w)), "nvfp4_device_error_word")
+    return int(w.value)

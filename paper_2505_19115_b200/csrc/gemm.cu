@@ -1,0 +1,471 @@
+// Block-scaled NVFP4 GEMM on the 5th-generation tensor cores (the contraction of Eq. 1-3):
+//   D[m,n] = (gA*gB) * sum_kb sA[m,kb]*sB[n,kb] * sum_{k in kb} a[m,k]*b[n,k]
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 0      TMA producer: packed codes by tiled bulk-tensor copies (128-byte swizzle), scale
+//               tiles by plain bulk copies, into a ring of shared-memory stages
+//   warp 1      MMA issuer: copies the stage's scales to tensor memory (tcgen05.cp) and issues
+//               tcgen05.mma kind::mxf4nvf4 (128 x BN x 64 per instruction), fp32 accumulators
+//               in tensor memory, double-buffered so the epilogue of tile i overlaps tile i+1
+//   warps 2..5  epilogue: tcgen05.ld the accumulator, scale by gA*gB, store fp32 or bf16
+// Every wait on an mbarrier is bounded in time; on a timeout the CTA records the site in a device
+// error word, drains its outstanding copies, frees its tensor memory and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace nvfp4 {
+namespace {
+
+__device__ unsigned int g_error_word = 0;
+
+constexpr int BM = 128;           // rows of A per tile (= UMMA M)
+constexpr int BK_BYTES = 128;     // packed bytes per row per stage = 256 E2M1 values
+constexpr int BK = 256;
+constexpr int MMA_K = 64;         // values per tcgen05.mma (32 bytes)
+constexpr int kGemmThreads = 192;
+constexpr uint32_t kTmemCols = 512;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+
+template <int BN>
+struct Cfg {
+  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kAccStages = (BN == 256) ? 1 : 2;
+  static constexpr int kABytes = BM * BK_BYTES;                   // 16 KB
+  static constexpr int kBBytes = BN * BK_BYTES;                   // 16 / 32 KB
+  static constexpr int kSfaBytes = 4 * 512;                       // 128 rows x 16 blocks
+  static constexpr int kSfbBytes = (BN / 128) * 4 * 512;
+  static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+  // tensor-memory columns: accumulators first, then two scale buffers (A: 16, B: BN/32*4 columns)
+  static constexpr uint32_t kAccCols = BN;
+  static constexpr uint32_t kSfaCol = kAccStages * BN;
+  static constexpr uint32_t kSfCols = 16 + (BN / 32) * 4;         // one stage of scales
+  static constexpr int kSfBufs = (kSfaCol + 2 * kSfCols <= kTmemCols) ? 2 : 1;
+  static_assert(kSfaCol + kSfBufs * kSfCols <= kTmemCols, "tensor memory overflow");
+};
+
+struct GemmParams {
+  const uint8_t* a_sf;
+  const uint8_t* b_sf;
+  const float* a_g;
+  const float* b_g;
+  void* d;
+  int64_t ldd;
+  int M, N, K;
+  int tiles_m, tiles_n, k_stages;   // k_stages = ceil(K / 256)
+  int k_tiles;                      // ceil(K / 64): 512-byte scale tiles per row tile
+  int a_row_tiles, b_row_tiles;     // ceil(M / 128), ceil(N / 128)
+  int d_is_bf16;
+};
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\t"
+               "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+               "selp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Returns false (and records `site`) if the barrier did not flip within the time
+// limit or another role of this CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
+  for (int i = 0; i < 2048; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  while (true) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_timer_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1u;
+      atomicOr(&g_error_word, 0x100u | site);
+      return false;
+    }
+    __nanosleep(128);
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 512 bytes of scales (32 rows x 16 bytes in shared memory) -> 4 tensor-memory columns, replicated
+// into all four 32-lane quarters.
+__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\t"
+               "setp.ne.b32 p, %4, 0;\n\t"
+               "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptors (64-bit): start address, leading/stride byte offsets (all >> 4),
+// descriptor version 1 at bit 46, swizzle mode at bits 61-63.
+// Operand tiles: K-major, 128-byte swizzle, rows 128 bytes apart, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+// Scale tile: 32 rows x 16 bytes, no swizzle, 8-row groups 128 bytes apart.
+__device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
+}
+// Instruction descriptor of kind::mxf4nvf4: E2M1 x E2M1 (format 1), K-major operands, UE4M3
+// scales, N >> 3 at bit 17, M >> 4 at bit 24.
+__host__ __device__ constexpr uint32_t instr_desc(int m, int n) {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (0u << 23) | ((uint32_t)(m >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------------
+// The kernel
+// ------------------------------------------------------------------------------------------------
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const GemmParams p) {
+  using C = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte aligned base for the swizzled operand tiles
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  // stage layout: [A 16K][B][SFA 2K][SFB]
+  const uint32_t bar_base = smem_base + C::kStages * C::kStageBytes;
+  uint8_t* bar_gen = smem_gen + C::kStages * C::kStageBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + C::kAccStages + a); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * C::kStages + 2 * C::kAccStages));
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < C::kAccStages; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 4); }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(smem_u32((const void*)tmem_slot), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer -------------------------------
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      uint32_t armed = 0, armed_ph = 0;  // per stage: armed at least once / phase of the last arming
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+        for (int ks = 0; ks < p.k_stages; ++ks) {
+          if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 1))) break;
+          const int kt0 = ks * 4;
+          const int nkt = min(4, p.k_tiles - kt0);                        // scale tiles in this stage
+          const uint32_t sf_bytes = (uint32_t)nkt * 512u;
+          const uint32_t st = smem_base + s * C::kStageBytes;
+          mbar_arrive_expect_tx(full_bar(s), C::kABytes + C::kBBytes + sf_bytes * (1 + BN / 128));
+          armed |= 1u << s;
+          armed_ph = (armed_ph & ~(1u << s)) | (ph << s);
+          tma_load_2d(st, &map_a, full_bar(s), ks * BK_BYTES, tm * BM);
+          tma_load_2d(st + C::kABytes, &map_b, full_bar(s), ks * BK_BYTES, tn * BN);
+          bulk_load(st + C::kABytes + C::kBBytes, p.a_sf + ((int64_t)tm * p.k_tiles + kt0) * 512, sf_bytes, full_bar(s));
+#pragma unroll
+          for (int h = 0; h < BN / 128; ++h) {
+            const int rt = min(tn * (BN / 128) + h, p.b_row_tiles - 1);   // clamp: rows past N are never stored
+            bulk_load(st + C::kABytes + C::kBBytes + C::kSfaBytes + h * 2048,
+                      p.b_sf + ((int64_t)rt * p.k_tiles + kt0) * 512, sf_bytes, full_bar(s));
+          }
+          if (++s == C::kStages) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // drain: give every armed stage a bounded chance to land before the CTA exits
+        for (int q = 0; q < C::kStages; ++q) {
+          if (!(armed & (1u << q))) continue;
+          const unsigned long long t0 = global_timer_ns();
+          while (!mbar_try_wait(full_bar(q), (armed_ph >> q) & 1u) && global_timer_ns() - t0 < 1000000ull) {}
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer -------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(BM, BN);
+      int s = 0;
+      uint32_t ph = 0;
+      int acc = 0;
+      uint32_t acc_ph = 0;
+      uint32_t sfbuf = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        if (!(ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, 2))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * C::kAccCols;
+        for (int ks = 0; ks < p.k_stages; ++ks) {
+          if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, 3))) break;
+          tc_fence_after();
+          const uint32_t st = smem_base + s * C::kStageBytes;
+          const int nkt = min(4, p.k_tiles - ks * 4);
+          const uint32_t sfa_t = tmem_base + C::kSfaCol + sfbuf * C::kSfCols;
+          const uint32_t sfb_t = sfa_t + 16;
+          for (int j = 0; j < nkt; ++j) {
+            tc_cp_sf(sfa_t + 4 * j, sf_desc(st + C::kABytes + C::kBBytes + 512 * j));
+#pragma unroll
+            for (int h = 0; h < BN / 128; ++h)
+              tc_cp_sf(sfb_t + (BN / 32) * j + 4 * h, sf_desc(st + C::kABytes + C::kBBytes + C::kSfaBytes + h * 2048 + 512 * j));
+          }
+          const uint64_t adesc = operand_desc(st), bdesc = operand_desc(st + C::kABytes);
+          for (int j = 0; j < nkt; ++j) {
+            tc_mma_nvf4(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, sfa_t + 4 * j, sfb_t + (BN / 32) * j,
+                        (ks | j) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(s));           // frees the stage once the MMAs above have read it
+          if (C::kSfBufs == 2) sfbuf ^= 1u;
+          if (++s == C::kStages) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));           // accumulator complete
+        if (++acc == C::kAccStages) { acc = 0; acc_ph ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------- epilogue -------------------------------
+    const int quarter = warp & 3;            // tensor-memory lanes this warp may read
+    const float alpha = (p.a_g ? __ldg(p.a_g) : 1.0f) * (p.b_g ? __ldg(p.b_g) : 1.0f);
+    int acc = 0;
+    uint32_t acc_ph = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+      const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+      if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, 4))) break;
+      tc_fence_after();
+      const int row = tm * BM + quarter * 32 + lane;
+      const uint32_t t_row = tmem_base + acc * C::kAccCols + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(t_row + c0, r);
+        tmem_ld_wait();
+        const int col = tn * BN + c0;
+        if (row < p.M && col < p.N) {
+          if (p.d_is_bf16) {
+            __nv_bfloat16* dst = static_cast<__nv_bfloat16*>(p.d) + (int64_t)row * p.ldd + col;
+            if (col + 32 <= p.N) {
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * v + 2 * e]) * alpha,
+                                                                 __uint_as_float(r[8 * v + 2 * e + 1]) * alpha);
+                  w[e] = *reinterpret_cast<const uint32_t*>(&h);
+                }
+                reinterpret_cast<uint4*>(dst)[v] = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            } else {
+              for (int e = 0; e < 32 && col + e < p.N; ++e) dst[e] = __float2bfloat16_rn(__uint_as_float(r[e]) * alpha);
+            }
+          } else {
+            float* dst = static_cast<float*>(p.d) + (int64_t)row * p.ldd + col;
+            if (col + 32 <= p.N) {
+#pragma unroll
+              for (int v = 0; v < 8; ++v)
+                reinterpret_cast<float4*>(dst)[v] =
+                    make_float4(__uint_as_float(r[4 * v]) * alpha, __uint_as_float(r[4 * v + 1]) * alpha,
+                                __uint_as_float(r[4 * v + 2]) * alpha, __uint_as_float(r[4 * v + 3]) * alpha);
+            } else {
+              for (int e = 0; e < 32 && col + e < p.N; ++e) dst[e] = __uint_as_float(r[e]) * alpha;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == C::kAccStages) { acc = 0; acc_ph ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// Packed codes [rows, row_bytes] -> box of (128 bytes x box_rows), 128-byte swizzle, zero fill.
+bool make_codes_map(CUtensorMap* map, const uint8_t* base, int64_t rows, int64_t row_bytes, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+  const cuuint32_t box[2] = {(cuuint32_t)BK_BYTES, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <int BN>
+int launch_gemm(const uint8_t* a_codes, const uint8_t* b_codes, GemmParams p, cudaStream_t s) {
+  using C = Cfg<BN>;
+  CUtensorMap map_a, map_b;
+  if (!make_codes_map(&map_a, a_codes, p.M, p.K / 2, BM)) return NVFP4_ERR_CUDA;
+  if (!make_codes_map(&map_b, b_codes, p.N, p.K / 2, BN)) return NVFP4_ERR_CUDA;
+  p.tiles_m = (p.M + BM - 1) / BM;
+  p.tiles_n = (p.N + BN - 1) / BN;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm_nvfp4_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
+      return NVFP4_ERR_CUDA;
+    attr_set = true;
+  }
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int grid = tiles < sm_count() ? tiles : sm_count();
+  gemm_nvfp4_kernel<BN><<<grid, kGemmThreads, C::kSmemBytes, s>>>(map_a, map_b, p);
+  return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+}  // namespace
+
+int gemm_tile_n_override = 0;  // 0 = automatic; 128 or 256 force a tile width (tuning/tests)
+
+}  // namespace nvfp4
+
+using namespace nvfp4;
+
+extern "C" int nvfp4_gemm_set_tile_n(int bn) {
+  if (bn != 0 && bn != 128 && bn != 256) return NVFP4_ERR_ENUM;
+  gemm_tile_n_override = bn;
+  return NVFP4_OK;
+}
+
+extern "C" int nvfp4_gemm(const uint8_t* a_codes, const uint8_t* a_sf, const float* a_g,
+                          const uint8_t* b_codes, const uint8_t* b_sf, const float* b_g,
+                          int64_t M, int64_t N, int64_t K, void* d, int d_dtype, int64_t ldd, void* cuda_stream) {
+  if (!a_codes || !a_sf || !b_codes || !b_sf || !d) return NVFP4_ERR_NULL;
+  if (d_dtype != NVFP4_BF16 && d_dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if (M <= 0 || N <= 0 || K <= 0 || (K % 32) != 0 || ldd < N) return NVFP4_ERR_SHAPE;
+  if (M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256 || K >= (1ll << 31) - 256) return NVFP4_ERR_SHAPE;
+  const int64_t esz = (d_dtype == NVFP4_BF16) ? 2 : 4;
+  if (!aligned16(a_codes) || !aligned16(a_sf) || !aligned16(b_codes) || !aligned16(b_sf) || !aligned16(d) ||
+      ((ldd * esz) % 16) != 0)
+    return NVFP4_ERR_ALIGN;
+  if ((a_g && (reinterpret_cast<uintptr_t>(a_g) & 3u)) || (b_g && (reinterpret_cast<uintptr_t>(b_g) & 3u)))
+    return NVFP4_ERR_ALIGN;
+  if (int st = check_arch()) return st;
+
+  GemmParams p;
+  p.a_sf = a_sf; p.b_sf = b_sf; p.a_g = a_g; p.b_g = b_g; p.d = d; p.ldd = ldd;
+  p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  p.k_stages = (int)ceil_div(K, BK);
+  p.k_tiles = (int)ceil_div(K, MMA_K);
+  p.a_row_tiles = (int)ceil_div(M, 128);
+  p.b_row_tiles = (int)ceil_div(N, 128);
+  p.d_is_bf16 = (d_dtype == NVFP4_BF16);
+  p.tiles_m = p.tiles_n = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  int bn = gemm_tile_n_override ? gemm_tile_n_override : 128;
+  return bn == 256 ? launch_gemm<256>(a_codes, b_codes, p, s) : launch_gemm<128>(a_codes, b_codes, p, s);
+}
+
+extern "C" int nvfp4_device_error_word(uint32_t* host_out) {
+  if (!host_out) return NVFP4_ERR_NULL;
+  unsigned int w = 0, zero = 0;
+  if (cudaMemcpyFromSymbol(&w, g_error_word, sizeof(w)) != cudaSuccess) return NVFP4_ERR_CUDA;
+  if (w != 0 && cudaMemcpyToSymbol(g_error_word, &zero, sizeof(zero)) != cudaSuccess) return NVFP4_ERR_CUDA;
+  *host_out = w;
+  return NVFP4_OK;
+}

@@ -1,0 +1,398 @@
+// NVFP4 quantizer kernels (Section 3 and Eq. 4-6 of the paper): block amax -> E4M3 scale ->
+// E2M1 codes with round-to-nearest or Philox stochastic rounding, along the contiguous axis
+// (row kernel) or along the row axis with a transposed output (transposed kernel), plus the
+// per-tensor amax scale.  All kernels are HBM-bound streaming kernels.
+#include <cuda_bf16.h>
+
+#include "common.cuh"
+
+namespace nvfp4 {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+struct QuantParams {
+  const void* x;
+  int64_t rows, cols, ld;
+  const float* gptr;
+  uint32_t seed_lo, seed_hi, off_lo, off_hi;
+  uint8_t* codes;
+  uint8_t* scales;
+  int64_t nkb;      // blocks per quantized row (Kq / 16)
+  int64_t k_tiles;  // ceil(nkb / 4)
+};
+
+// One block of 16 values -> 8 bytes of codes (lo, hi words) and one scale byte.
+// c = (1/6)/g, g = per-tensor scale.  `blk` is the block's linear index (Philox counter).
+template <bool SR>
+__device__ __forceinline__ void quantize_block(const float (&v)[16], float c, float g,
+                                               const QuantParams& p, uint64_t blk,
+                                               uint32_t& lo, uint32_t& hi, uint32_t& sf) {
+  float amax = 0.0f;
+#pragma unroll
+  for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(v[j]));
+  const uint32_t q = e4m3_encode(__fmul_rn(amax, c));
+  const float d = __fmul_rn(e4m3_decode(q), g);
+  const float inv = (q == 0u) ? 0.0f : __fdiv_rn(1.0f, d);
+  sf = q;
+  uint32_t w[2] = {0u, 0u};
+  if constexpr (!SR) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float y0 = fminf(__fmul_rn(fabsf(v[2 * j]), inv), 6.0f);
+      const float y1 = fminf(__fmul_rn(fabsf(v[2 * j + 1]), inv), 6.0f);
+      uint32_t b = e2m1x2_rn(y0, y1);
+      b |= ((__float_as_uint(v[2 * j]) >> 28) & 0x8u) | ((__float_as_uint(v[2 * j + 1]) >> 24) & 0x80u);
+      w[j >> 2] |= b << (8 * (j & 3));
+    }
+  } else {
+    const uint4 r4 = philox4x32_10(p.seed_lo, p.seed_hi, (uint32_t)blk, (uint32_t)(blk >> 32), p.off_lo, p.off_hi);
+    const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const uint32_t u = (rw[j >> 2] >> (8 * (j & 3))) & 0xFFu;
+      const float y = fminf(__fmul_rn(fabsf(v[j]), inv), 6.0f);
+      const uint32_t nib = e2m1_sr(y, u) | ((__float_as_uint(v[j]) >> 28) & 0x8u);
+      w[j >> 3] |= nib << (4 * (j & 7));
+    }
+  }
+  lo = w[0];
+  hi = w[1];
+}
+
+__device__ __forceinline__ void unpack_bf16x8(const uint4& q, float* v) {
+  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void load_block16(const T* src, float (&v)[16]) {
+  if constexpr (sizeof(T) == 2) {
+    const uint4 a = __ldg(reinterpret_cast<const uint4*>(src));
+    const uint4 b = __ldg(reinterpret_cast<const uint4*>(src) + 1);
+    unpack_bf16x8(a, v);
+    unpack_bf16x8(b, v + 8);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 f = __ldg(reinterpret_cast<const float4*>(src) + i);
+      v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+    }
+  }
+}
+
+// -------------------------------------------------------------------------------------------------
+// Row quantizer: CTA tile = 128 rows x 32 blocks (512 columns); warp w takes rows w, w+8, ...;
+// lane = block within the row segment, so a warp reads 1 KB (bf16) of one row per step and
+// writes 256 contiguous code bytes.  Swizzled scales are staged in shared memory and leave as
+// eight contiguous 512-byte tiles.
+// -------------------------------------------------------------------------------------------------
+constexpr int kRowTileRows = 128;
+constexpr int kSfChunkPitch = 528;  // 512 + 16: spreads the eight k-tiles over different banks
+
+template <typename T, bool SR, bool SWZ>
+__global__ void __launch_bounds__(kThreads) quantize_row_kernel(const QuantParams p) {
+  __shared__ __align__(16) uint8_t sf_s[SWZ ? 8 * kSfChunkPitch : 16];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t kb = (int64_t)blockIdx.x * 32 + lane;
+  const int64_t row0 = (int64_t)blockIdx.y * kRowTileRows;
+  const bool kb_ok = kb < p.nkb;
+  const float g = p.gptr ? __ldg(p.gptr) : 1.0f;
+  const float c = __fdiv_rn(__fdiv_rn(1.0f, 6.0f), g);
+  const T* x = static_cast<const T*>(p.x);
+
+  if constexpr (SWZ) {
+    for (int i = threadIdx.x; i < 8 * kSfChunkPitch / 16; i += kThreads)
+      reinterpret_cast<uint4*>(sf_s)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+  }
+
+  constexpr int U = 4;  // rows in flight per thread
+#pragma unroll 1
+  for (int it = 0; it < kRowTileRows / 8; it += U) {
+    float v[U][16];
+    bool ok[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int64_t r = row0 + warp + 8 * (it + u);
+      ok[u] = kb_ok && r < p.rows;
+      if (ok[u]) load_block16<T>(x + r * p.ld + kb * 16, v[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (!ok[u]) continue;
+      const int rl = warp + 8 * (it + u);
+      const int64_t r = row0 + rl;
+      uint32_t lo, hi, sf;
+      quantize_block<SR>(v[u], c, g, p, (uint64_t)(r * p.nkb + kb), lo, hi, sf);
+      *reinterpret_cast<uint2*>(p.codes + (r * p.nkb + kb) * 8) = make_uint2(lo, hi);
+      if constexpr (SWZ) {
+        sf_s[(lane >> 2) * kSfChunkPitch + (rl & 31) * 16 + (rl >> 5) * 4 + (lane & 3)] = (uint8_t)sf;
+      } else {
+        p.scales[r * p.nkb + kb] = (uint8_t)sf;
+      }
+    }
+  }
+
+  if constexpr (SWZ) {
+    __syncthreads();
+    const int q = threadIdx.x >> 5, i = threadIdx.x & 31;
+    const int64_t kt = (int64_t)blockIdx.x * 8 + q;
+    if (kt < p.k_tiles) {
+      const uint4 val = *reinterpret_cast<const uint4*>(sf_s + q * kSfChunkPitch + i * 16);
+      *reinterpret_cast<uint4*>(p.scales + ((int64_t)blockIdx.y * p.k_tiles + kt) * 512 + i * 16) = val;
+    }
+  }
+}
+
+// -------------------------------------------------------------------------------------------------
+// Transposed quantizer: blocks run along the row axis of x[rows, cols]; the output is stored as
+// [cols, rows/2] codes and [cols, rows/16] scales.  A CTA stages a (TILE_R rows x 64 cols) tile
+// in shared memory with 16-byte async copies (zero-filled outside the tensor), every thread
+// quantizes column pairs from it, and codes/scales leave through a second staging buffer so
+// that global stores run along the output's contiguous axis.
+// -------------------------------------------------------------------------------------------------
+constexpr int kTCols = 64;
+
+__device__ __forceinline__ void cp_async16_zfill(void* smem_dst, const void* gsrc, int src_bytes) {
+  const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+
+template <typename T>
+struct TTile {
+  static constexpr int kRows = (sizeof(T) == 2) ? 256 : 128;          // 32 KB of input per tile
+  static constexpr int kRowBlocks = kRows / 16;                        // 16 or 8
+  static constexpr int kCodePitch = kRows / 2 + 8;                     // bytes per staged output row
+  static constexpr int kChunksPerRow = kTCols * (int)sizeof(T) / 16;   // 8 or 16
+};
+
+template <typename T, bool SR, bool SWZ>
+__global__ void __launch_bounds__(kThreads) quantize_transposed_kernel(const QuantParams p) {
+  using TT = TTile<T>;
+  extern __shared__ __align__(16) uint8_t smem[];
+  T* tile = reinterpret_cast<T*>(smem);                                        // [kRows][64]
+  uint8_t* code_s = smem + TT::kRows * kTCols * sizeof(T);                     // [64][kCodePitch]
+  uint8_t* sf_s = code_s + kTCols * TT::kCodePitch;                            // [64][kRowBlocks]
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t c0 = (int64_t)blockIdx.x * kTCols;
+  const int64_t r0 = (int64_t)blockIdx.y * TT::kRows;
+  const T* x = static_cast<const T*>(p.x);
+  const float g = p.gptr ? __ldg(p.gptr) : 1.0f;
+  const float c = __fdiv_rn(__fdiv_rn(1.0f, 6.0f), g);
+
+  // ---- stage the input tile ----
+  constexpr int kElemsPerChunk = 16 / (int)sizeof(T);
+  constexpr int kChunks = TT::kRows * TT::kChunksPerRow;
+#pragma unroll
+  for (int i = 0; i < kChunks / kThreads; ++i) {
+    const int id = threadIdx.x + i * kThreads;
+    const int row = id / TT::kChunksPerRow, ch = id % TT::kChunksPerRow;
+    const int64_t gr = r0 + row, gc = c0 + (int64_t)ch * kElemsPerChunk;
+    int64_t valid = (gr < p.rows) ? (p.cols - gc) : 0;
+    valid = valid < 0 ? 0 : (valid > kElemsPerChunk ? kElemsPerChunk : valid);
+    const T* src = (valid > 0) ? (x + gr * p.ld + gc) : x;
+    cp_async16_zfill(tile + row * kTCols + ch * kElemsPerChunk, src, (int)valid * (int)sizeof(T));
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  // ---- quantize: lane -> columns (2*lane, 2*lane+1), warp -> row blocks ----
+#pragma unroll 1
+  for (int rb = warp; rb < TT::kRowBlocks; rb += kThreads / 32) {
+    float va[16], vb[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const T* e = tile + (rb * 16 + j) * kTCols + 2 * lane;
+      if constexpr (sizeof(T) == 2) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(e);
+        va[j] = __uint_as_float(w << 16);
+        vb[j] = __uint_as_float(w & 0xFFFF0000u);
+      } else {
+        const float2 f = *reinterpret_cast<const float2*>(e);
+        va[j] = f.x;
+        vb[j] = f.y;
+      }
+    }
+    const int64_t kb = r0 / 16 + rb;
+    const int64_t ca = c0 + 2 * lane;
+    uint32_t lo, hi, sf;
+    quantize_block<SR>(va, c, g, p, (uint64_t)(ca * p.nkb + kb), lo, hi, sf);
+    *reinterpret_cast<uint2*>(code_s + (2 * lane) * TT::kCodePitch + rb * 8) = make_uint2(lo, hi);
+    sf_s[(2 * lane) * TT::kRowBlocks + rb] = (uint8_t)sf;
+    quantize_block<SR>(vb, c, g, p, (uint64_t)((ca + 1) * p.nkb + kb), lo, hi, sf);
+    *reinterpret_cast<uint2*>(code_s + (2 * lane + 1) * TT::kCodePitch + rb * 8) = make_uint2(lo, hi);
+    sf_s[(2 * lane + 1) * TT::kRowBlocks + rb] = (uint8_t)sf;
+  }
+  __syncthreads();
+
+  // ---- codes out: 8-byte units, contiguous along the quantized row ----
+  const int64_t kb0 = r0 / 16;
+#pragma unroll
+  for (int i = 0; i < kTCols * TT::kRowBlocks / kThreads; ++i) {
+    const int id = threadIdx.x + i * kThreads;
+    const int cl = id / TT::kRowBlocks, u = id % TT::kRowBlocks;
+    if (c0 + cl < p.cols && kb0 + u < p.nkb) {
+      const uint2 val = *reinterpret_cast<const uint2*>(code_s + cl * TT::kCodePitch + u * 8);
+      *reinterpret_cast<uint2*>(p.codes + ((c0 + cl) * p.nkb + kb0 + u) * 8) = val;
+    }
+  }
+  // ---- scales out ----
+  if constexpr (SWZ) {
+    constexpr int kKt = TT::kRowBlocks / 4;  // k-tiles per CTA tile
+    const bool fill_upper = ((c0 & 127) == 0) && (c0 + kTCols >= p.cols);  // nobody else owns rows 64..127
+    for (int id = threadIdx.x; id < kTCols * kKt; id += kThreads) {
+      const int cl = id / kKt, t = id % kKt;
+      const int64_t kt = kb0 / 4 + t;
+      if (kt >= p.k_tiles) continue;
+      const uint32_t val = *reinterpret_cast<const uint32_t*>(sf_s + cl * TT::kRowBlocks + t * 4);
+      *reinterpret_cast<uint32_t*>(p.scales + sf_swizzled_offset(c0 + cl, kt * 4, p.k_tiles)) = val;
+      if (fill_upper)
+        *reinterpret_cast<uint32_t*>(p.scales + sf_swizzled_offset(c0 + cl + 64, kt * 4, p.k_tiles)) = 0u;
+    }
+  } else {
+    for (int id = threadIdx.x; id < kTCols * TT::kRowBlocks; id += kThreads) {
+      const int cl = id / TT::kRowBlocks, u = id % TT::kRowBlocks;
+      if (c0 + cl < p.cols && kb0 + u < p.nkb) p.scales[(c0 + cl) * p.nkb + kb0 + u] = sf_s[id];
+    }
+  }
+}
+
+// -------------------------------------------------------------------------------------------------
+// Per-tensor amax -> g = amax / (6*448)
+// -------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kThreads) amax_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld,
+                                                        unsigned int* out_bits) {
+  constexpr int kVec = 16 / (int)sizeof(T);
+  const int64_t vec_per_row = cols / kVec;
+  const int64_t total = rows * vec_per_row;
+  float amax = 0.0f;
+  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < total; i += (int64_t)gridDim.x * kThreads) {
+    const int64_t r = i / vec_per_row, vcol = i % vec_per_row;
+    const uint4 q = __ldg(reinterpret_cast<const uint4*>(x + r * ld + vcol * kVec));
+    if constexpr (sizeof(T) == 2) {
+      float v[8];
+      unpack_bf16x8(q, v);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(v[j]));
+    } else {
+      amax = fmaxf(fmaxf(fabsf(__uint_as_float(q.x)), fabsf(__uint_as_float(q.y))),
+                   fmaxf(fmaxf(fabsf(__uint_as_float(q.z)), fabsf(__uint_as_float(q.w))), amax));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+  if ((threadIdx.x & 31) == 0 && amax > 0.0f) atomicMax(out_bits, __float_as_uint(amax));  // non-negative floats order as ints
+}
+
+__global__ void amax_finalize_kernel(float* out) {
+  const float amax = *out;
+  *out = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 2688.0f);
+}
+
+template <typename T, bool SR, bool SWZ>
+cudaError_t launch_row(const QuantParams& p, cudaStream_t s) {
+  dim3 grid((unsigned)ceil_div(p.nkb, 32), (unsigned)ceil_div(p.rows, kRowTileRows));
+  quantize_row_kernel<T, SR, SWZ><<<grid, kThreads, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+template <typename T, bool SR, bool SWZ>
+cudaError_t launch_transposed(const QuantParams& p, cudaStream_t s) {
+  using TT = TTile<T>;
+  const size_t smem = TT::kRows * kTCols * sizeof(T) + kTCols * TT::kCodePitch + kTCols * TT::kRowBlocks;
+  static bool attr_set = false;  // one attribute per instantiation; harmless if repeated
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(quantize_transposed_kernel<T, SR, SWZ>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  dim3 grid((unsigned)ceil_div(p.cols, kTCols), (unsigned)ceil_div(p.rows, TT::kRows));
+  quantize_transposed_kernel<T, SR, SWZ><<<grid, kThreads, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+template <typename T>
+cudaError_t dispatch(const QuantParams& p, bool transposed, bool sr, bool swz, cudaStream_t s) {
+  if (!transposed) {
+    if (sr) return swz ? launch_row<T, true, true>(p, s) : launch_row<T, true, false>(p, s);
+    return swz ? launch_row<T, false, true>(p, s) : launch_row<T, false, false>(p, s);
+  }
+  if (sr) return swz ? launch_transposed<T, true, true>(p, s) : launch_transposed<T, true, false>(p, s);
+  return swz ? launch_transposed<T, false, true>(p, s) : launch_transposed<T, false, false>(p, s);
+}
+
+}  // namespace
+
+}  // namespace nvfp4
+
+using namespace nvfp4;
+
+extern "C" size_t nvfp4_sf_bytes(int64_t Rq, int64_t Kq, int sf_layout) {
+  if (Rq <= 0 || Kq <= 0 || (Kq % 16) != 0) return 0;
+  if (sf_layout == NVFP4_SF_LINEAR) return (size_t)(Rq * (Kq / 16));
+  if (sf_layout == NVFP4_SF_SWIZZLED_128x4) return (size_t)(ceil_div(Rq, 128) * ceil_div(Kq, 64) * 512);
+  return 0;
+}
+
+extern "C" int nvfp4_quantize(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                              int transposed, const float* global_scale, const nvfp4_rounding* rounding,
+                              uint8_t* codes, uint8_t* scales, int sf_layout, void* cuda_stream) {
+  if (!x || !rounding || !codes || !scales) return NVFP4_ERR_NULL;
+  if (dtype != NVFP4_BF16 && dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if (transposed != 0 && transposed != 1) return NVFP4_ERR_ENUM;
+  if (rounding->mode != NVFP4_RTN && rounding->mode != NVFP4_SR) return NVFP4_ERR_ENUM;
+  if (rounding->reserved != 0) return NVFP4_ERR_ENUM;
+  if (sf_layout != NVFP4_SF_LINEAR && sf_layout != NVFP4_SF_SWIZZLED_128x4) return NVFP4_ERR_ENUM;
+  if (rows <= 0 || cols <= 0 || ld < cols) return NVFP4_ERR_SHAPE;
+  const int64_t Kq = transposed ? rows : cols;
+  if (Kq % 16 != 0 || cols % 8 != 0) return NVFP4_ERR_SHAPE;
+  if (rows >= (int64_t)1 << 31 || cols >= (int64_t)1 << 31) return NVFP4_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(codes) || !aligned16(scales) || (ld % 8) != 0) return NVFP4_ERR_ALIGN;
+  if (int st = check_arch()) return st;
+
+  QuantParams p;
+  p.x = x; p.rows = rows; p.cols = cols; p.ld = ld; p.gptr = global_scale;
+  p.seed_lo = (uint32_t)rounding->seed; p.seed_hi = (uint32_t)(rounding->seed >> 32);
+  p.off_lo = (uint32_t)rounding->offset; p.off_hi = (uint32_t)(rounding->offset >> 32);
+  p.codes = codes; p.scales = scales;
+  p.nkb = Kq / 16; p.k_tiles = ceil_div(p.nkb, 4);
+  if (ceil_div(rows, 128) > 65535) return NVFP4_ERR_SHAPE;  // grid.y limit
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const bool sr = rounding->mode == NVFP4_SR, swz = sf_layout == NVFP4_SF_SWIZZLED_128x4;
+  cudaError_t e = (dtype == NVFP4_BF16) ? dispatch<__nv_bfloat16>(p, transposed != 0, sr, swz, s)
+                                        : dispatch<float>(p, transposed != 0, sr, swz, s);
+  return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+extern "C" int nvfp4_tensor_amax_scale(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                                       float* global_scale_out, void* cuda_stream) {
+  if (!x || !global_scale_out) return NVFP4_ERR_NULL;
+  if (dtype != NVFP4_BF16 && dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if (rows <= 0 || cols <= 0 || ld < cols || cols % 8 != 0) return NVFP4_ERR_SHAPE;
+  if (!aligned16(x) || (ld % 8) != 0 || (reinterpret_cast<uintptr_t>(global_scale_out) & 3u)) return NVFP4_ERR_ALIGN;
+  if (int st = check_arch()) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaMemsetAsync(global_scale_out, 0, sizeof(float), s) != cudaSuccess) return NVFP4_ERR_CUDA;
+  const int64_t vecs = rows * (cols / (dtype == NVFP4_BF16 ? 8 : 4));
+  int64_t blocks = ceil_div(vecs, (int64_t)kThreads * 4);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks < 1) blocks = 1;
+  unsigned int* bits = reinterpret_cast<unsigned int*>(global_scale_out);
+  if (dtype == NVFP4_BF16)
+    amax_kernel<__nv_bfloat16><<<(unsigned)blocks, kThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(x), rows, cols, ld, bits);
+  else
+    amax_kernel<float><<<(unsigned)blocks, kThreads, 0, s>>>(static_cast<const float*>(x), rows, cols, ld, bits);
+  if (cudaGetLastError() != cudaSuccess) return NVFP4_ERR_CUDA;
+  amax_finalize_kernel<<<1, 1, 0, s>>>(global_scale_out);
+  return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}

@@ -1,0 +1,125 @@
+"""GPU-vs-oracle parity of the block-scaled GEMM: |gpu - oracle| <= 1e-5 * sum|a_i b_i| elementwise,
+exact equality where every partial sum is exactly representable."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import binding as ob
+from paper_2505_19115_b200 import binding as nb
+from paper_2505_19115_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+
+
+def _quantized_pair(M, N, K, seed, a_std=1.0, b_std=0.02, use_g=True, sr=False):
+    A = synth.normal((M, K), a_std, seed, device="cpu").cuda()
+    B = synth.normal((N, K), b_std, seed + 1, device="cpu").cuda()
+    ga = nb.nvfp4_tensor_amax_scale(A) if use_g else None
+    gb = nb.nvfp4_tensor_amax_scale(B) if use_g else None
+    r = nb.Rounding(nb.SR, 3, 1) if sr else nb.Rounding()
+    ac, asf = nb.nvfp4_quantize(A, global_scale=ga, rounding=r, sf_layout=nb.SF_SWIZZLED)
+    bc, bsf = nb.nvfp4_quantize(B, global_scale=gb, rounding=r, sf_layout=nb.SF_SWIZZLED)
+    # the oracle consumes linear scales produced by the oracle's own quantizer (bit-identical
+    # to the GPU's, which the quantizer parity tests establish)
+    gaf = float(ga.item()) if use_g else 1.0
+    gbf = float(gb.item()) if use_g else 1.0
+    oac, oasf = ob.quantize(A.float().cpu().numpy(), g=gaf, mode=r.mode, seed=r.seed, offset=r.offset)
+    obc, obsf = ob.quantize(B.float().cpu().numpy(), g=gbf, mode=r.mode, seed=r.seed, offset=r.offset)
+    assert np.array_equal(oac, ac.cpu().numpy()) and np.array_equal(obc, bc.cpu().numpy())
+    return (ac, asf, ga, bc, bsf, gb), (oac, oasf, gaf, obc, obsf, gbf)
+
+
+def _check(gpu_ops, ora_ops, out_dtype=torch.float32):
+    D = nb.nvfp4_gemm(*gpu_ops, out_dtype=out_dtype)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
+    ref, T = ob.gemm(*ora_ops)
+    got = D.float().cpu().numpy()
+    if out_dtype == torch.bfloat16:
+        assert np.all(np.abs(got - ref) <= TOL * T + np.abs(ref) * 2.0 ** -8)
+    else:
+        err = np.abs(got - ref)
+        bad = np.argwhere(err > TOL * T)
+        assert bad.size == 0, f"{bad.shape[0]} of {err.size} outputs beyond tolerance, first {bad[:3]}, " \
+                              f"max ratio {np.max(err / np.maximum(T, 1e-30)):.3e}"
+    return got, ref
+
+
+@pytest.fixture(params=[128, 256])
+def tile_n(request):
+    nb.nvfp4_gemm_set_tile_n(request.param)
+    yield request.param
+    nb.nvfp4_gemm_set_tile_n(0)
+
+
+def test_one_hot_rows_read_back_dequantized_operand(tile_n):
+    # A row with a single 6.0 (scale 1, code 7) selects one column of dequantized B: any error in
+    # the scale-tile layout, the operand descriptors or the nibble order shows up exactly.
+    M, N, K = 256, 384, 512
+    A = torch.zeros((M, K), dtype=torch.float32)
+    for m in range(M):
+        A[m, (m * 37) % K] = 6.0
+    B = synth.normal((N, K), 1.0, 5, device="cpu").float()
+    ac, asf = nb.nvfp4_quantize(A.cuda(), sf_layout=nb.SF_SWIZZLED)
+    bc, bsf = nb.nvfp4_quantize(B.cuda(), sf_layout=nb.SF_SWIZZLED)
+    D = nb.nvfp4_gemm(ac, asf, None, bc, bsf, None).cpu().numpy()
+    assert nb.nvfp4_device_error_word() == 0
+    obc, obsf = ob.quantize(B.numpy())
+    deqB = ob.dequantize(obc, obsf)
+    want = np.stack([6.0 * deqB[:, (m * 37) % K] for m in range(M)])
+    assert np.array_equal(D, want)
+
+
+def test_exact_when_all_partial_sums_are_representable(tile_n):
+    rng = np.random.default_rng(0)
+    grid = np.array([0, 0.5, 1, 1.5, 2, 3, 4, 6, -0.5, -1, -1.5, -2, -3, -4, -6], dtype=np.float32)
+    M, N, K = 128, 256, 256
+    A = rng.choice(grid, size=(M, K)).astype(np.float32)
+    B = rng.choice(grid, size=(N, K)).astype(np.float32)
+    A[:, ::16] = 6.0
+    B[:, ::16] = -6.0                                  # every block has amax 6 -> scale exactly 1
+    ac, asf = nb.nvfp4_quantize(torch.from_numpy(A).cuda(), sf_layout=nb.SF_SWIZZLED)
+    bc, bsf = nb.nvfp4_quantize(torch.from_numpy(B).cuda(), sf_layout=nb.SF_SWIZZLED)
+    D = nb.nvfp4_gemm(ac, asf, None, bc, bsf, None).cpu().numpy()
+    assert np.array_equal(D, (A.astype(np.float64) @ B.astype(np.float64).T).astype(np.float32))
+
+
+@pytest.mark.parametrize("shape", [(128, 128, 256), (256, 256, 512), (130, 136, 320), (257, 392, 1056),
+                                   (1, 8, 32), (64, 200, 96), (384, 520, 2080)])
+def test_random_operands_within_tolerance(shape, tile_n):
+    M, N, K = shape
+    gpu_ops, ora_ops = _quantized_pair(M, N, K, seed=10 + M)
+    _check(gpu_ops, ora_ops)
+
+
+def test_stochastically_rounded_operands_and_no_global_scale(tile_n):
+    gpu_ops, ora_ops = _quantized_pair(256, 256, 512, seed=40, b_std=1.0, use_g=False, sr=True)
+    _check(gpu_ops, ora_ops)
+
+
+def test_bf16_output(tile_n):
+    gpu_ops, ora_ops = _quantized_pair(256, 256, 512, seed=50)
+    _check(gpu_ops, ora_ops, out_dtype=torch.bfloat16)
+
+
+@pytest.mark.parametrize("K", [64, 256, 1024, 4096, 16384, 65536])
+def test_error_stays_under_tolerance_as_K_grows(K):
+    # detects reduced-precision accumulation in the tensor core: the oracle accumulates in double
+    gpu_ops, ora_ops = _quantized_pair(128, 128, K, seed=60, b_std=1.0)
+    got, ref = _check(gpu_ops, ora_ops)
+
+
+def test_many_tiles_persistent_schedule():
+    # more tiles than SMs, ragged edges in both directions
+    gpu_ops, ora_ops = _quantized_pair(2000, 2600, 512, seed=70)
+    D = nb.nvfp4_gemm(*gpu_ops)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
+    rng = np.random.default_rng(1)
+    ii = np.concatenate([rng.integers(0, 2000, 4096), np.full(2600, 1999), np.arange(2000)])
+    jj = np.concatenate([rng.integers(0, 2600, 4096), np.arange(2600), np.full(2000, 2599)])
+    ref, T = ob.gemm_sampled(*ora_ops, ii, jj)
+    got = D.cpu().numpy()[ii, jj]
+    assert np.all(np.abs(got - ref) <= TOL * T)

@@ -1,0 +1,116 @@
+"""GPU-vs-oracle parity of the three quantized linear-layer products (Eq. 1-6)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import binding as ob
+from paper_2505_19115_b200 import binding as nb
+from paper_2505_19115_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+
+
+def _host(x):
+    return x.float().cpu().numpy()
+
+
+def _oracle_operand(x, transposed, r, use_g):
+    h = _host(x)
+    g = ob.tensor_amax_scale(h) if use_g else 1.0
+    c, s = ob.quantize(h, g=g, mode=r.mode, seed=r.seed, offset=r.offset, transposed=transposed)
+    return c, s, g
+
+
+def oracle_linear(which, a, b, ra, rb, use_g, sample=None):
+    ta, tb = {"fwd": (False, False), "dx": (False, True), "dw": (True, True)}[which]
+    ac, asf, ga = _oracle_operand(a, ta, ra, use_g)
+    bc, bsf, gb = _oracle_operand(b, tb, rb, use_g)
+    if sample is None:
+        return ob.gemm(ac, asf, ga, bc, bsf, gb)
+    return ob.gemm_sampled(ac, asf, ga, bc, bsf, gb, sample[0], sample[1])
+
+
+def _assert_close(got, ref, T):
+    err = np.abs(got - ref)
+    assert np.all(err <= TOL * T), f"max err/T = {np.max(err / np.maximum(T, 1e-30)):.3e}"
+
+
+@pytest.mark.parametrize("use_g", [True, False])
+def test_single_layer_all_three_products(use_g):
+    # single small layer: X 256x512 N(0,1), W 512x512 N(0,0.02^2), dY 256x512 N(0,1e-3^2)
+    t = synth.TINY_LINEAR
+    X, W, dY = synth.linear_inputs(t["tokens"], t["K"], t["N"], seed=1001, grad_std=1e-3)
+    X, W, dY = X.cuda(), W.cuda(), dY.cuda()
+    mode = nb.G_AMAX if use_g else nb.G_NONE
+    rt, sr0, sr1, sr2 = nb.Rounding(nb.RTN), nb.Rounding(nb.SR, 0, 0), nb.Rounding(nb.SR, 0, 1), nb.Rounding(nb.SR, 0, 2)
+    Y = nb.nvfp4_linear_fwd(X, W, gscale_mode=mode, rx=rt, rw=rt)
+    dX = nb.nvfp4_linear_bwd_dx(dY, W, gscale_mode=mode, rdy=sr0, rw=rt)
+    dW = nb.nvfp4_linear_bwd_dw(dY, X, gscale_mode=mode, rdy=sr1, rx=sr2)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
+    _assert_close(_host(Y), *oracle_linear("fwd", X, W, rt, rt, use_g))
+    _assert_close(_host(dX), *oracle_linear("dx", dY, W, sr0, rt, use_g))
+    _assert_close(_host(dW), *oracle_linear("dw", dY, X, sr1, sr2, use_g))
+    if not use_g:
+        # without a per-tensor scale the 1e-3 gradients underflow the E4M3 scale range entirely
+        assert float(dX.abs().max()) == 0.0 and float(dW.abs().max()) == 0.0
+    else:
+        assert float(dX.abs().max()) > 0.0 and float(dW.abs().max()) > 0.0
+
+
+def test_all_sr_backward_variant():
+    # the single-layer config also asks for SR on W in the backward product
+    t = synth.TINY_LINEAR
+    X, W, dY = synth.linear_inputs(t["tokens"], t["K"], t["N"], seed=1001, grad_std=1e-3)
+    W, dY = W.cuda(), dY.cuda()
+    sr0, sr3 = nb.Rounding(nb.SR, 0, 0), nb.Rounding(nb.SR, 0, 3)
+    dX = nb.nvfp4_linear_bwd_dx(dY, W, rdy=sr0, rw=sr3)
+    _assert_close(_host(dX), *oracle_linear("dx", dY, W, sr0, sr3, True))
+
+
+def test_ragged_layer_and_bf16_output():
+    X, W, dY = synth.linear_inputs(160, 288, 200, seed=7, grad_std=1e-3)
+    X, W, dY = X.cuda(), W.cuda(), dY.cuda()
+    rt, sr = nb.Rounding(nb.RTN), nb.Rounding(nb.SR, 9, 0)
+    Y = nb.nvfp4_linear_fwd(X, W, rx=rt, rw=rt)
+    _assert_close(_host(Y), *oracle_linear("fwd", X, W, rt, rt, True))
+    dW = nb.nvfp4_linear_bwd_dw(dY, X, rdy=sr, rx=sr)
+    _assert_close(_host(dW), *oracle_linear("dw", dY, X, sr, sr, True))
+    Yb = nb.nvfp4_linear_fwd(X, W, rx=rt, rw=rt, out_dtype=torch.bfloat16)
+    ref, T = oracle_linear("fwd", X, W, rt, rt, True)
+    assert np.all(np.abs(_host(Yb) - ref) <= TOL * T + np.abs(ref) * 2.0 ** -8)
+
+
+def test_given_global_scales_and_fp32_inputs():
+    X, W, _ = synth.linear_inputs(128, 256, 128, seed=8)
+    X, W = X.float().cuda(), W.float().cuda()
+    gx, gw = nb.nvfp4_tensor_amax_scale(X), nb.nvfp4_tensor_amax_scale(W)
+    rt = nb.Rounding(nb.RTN)
+    Y = nb.nvfp4_linear_fwd(X, W, gscale_mode=nb.G_GIVEN, gx=gx, gw=gw, rx=rt, rw=rt)
+    _assert_close(_host(Y), *oracle_linear("fwd", X, W, rt, rt, True))
+
+
+@pytest.mark.parametrize("name,K,N", [(n, k, o) for (n, k, o) in synth.LLAMA_350M["linears"] if n in ("qkv", "down")])
+def test_350m_block_linears_sampled(name, K, N):
+    M = synth.LLAMA_350M["tokens"]
+    X, W, dY = synth.linear_inputs(M, K, N, seed=1003)
+    X, W, dY = X.cuda(), W.cuda(), dY.cuda()
+    rt, sr0, sr1, sr2 = nb.Rounding(nb.RTN), nb.Rounding(nb.SR, 0, 0), nb.Rounding(nb.SR, 0, 1), nb.Rounding(nb.SR, 0, 2)
+    rng = np.random.default_rng(3)
+    n = 2048
+
+    def sample(R, C):
+        return (np.concatenate([rng.integers(0, R, n), [0, R - 1]]), np.concatenate([rng.integers(0, C, n), [C - 1, 0]]))
+
+    Y = nb.nvfp4_linear_fwd(X, W, rx=rt, rw=rt)
+    s = sample(M, N)
+    _assert_close(_host(Y)[s[0], s[1]], *oracle_linear("fwd", X, W, rt, rt, True, s))
+    dX = nb.nvfp4_linear_bwd_dx(dY, W, rdy=sr0, rw=rt)
+    s = sample(M, K)
+    _assert_close(_host(dX)[s[0], s[1]], *oracle_linear("dx", dY, W, sr0, rt, True, s))
+    dW = nb.nvfp4_linear_bwd_dw(dY, X, rdy=sr1, rx=sr2)
+    s = sample(N, K)
+    _assert_close(_host(dW)[s[0], s[1]], *oracle_linear("dw", dY, X, sr1, sr2, True, s))
+    assert nb.nvfp4_device_error_word() == 0
