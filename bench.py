@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the NVFP4 quantize-then-GEMM hot path on B200.
+
+One "step" is one pass of the whole hot path over one Llama-7B-shaped transformer block's five
+linear layers (tokens 16384, hidden 4096): for each layer the forward product (Eq. 1/4), the
+input-gradient product (Eq. 2/5) and the weight-gradient product (Eq. 3/6), each with its
+per-tensor amax passes, its two operand quantizations and its block-scaled GEMM, all through
+the C-ABI entry points nvfp4_linear_fwd / nvfp4_linear_bwd_dx / nvfp4_linear_bwd_dw.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample of
+the same workload instead.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2505_19115_b200 import synth  # noqa: E402
+
+METRIC = "NVFP4 linear fwd+bwd TFLOPS (% FP4 peak); quantizer GB/s (% HBM peak)"
+FP4_OVER_BF16 = 4.0        # nominal dense ratio: 9 PFLOP/s NVFP4 vs 2.25 PFLOP/s bf16
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram bytes per GEMM launch from the committed ncu capture (profiles/); None until measured
+GEMM_TRAFFIC_BYTES = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def block_flops(cfg):
+    return sum(6.0 * cfg["tokens"] * K * N for _, K, N in cfg["linears"])
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.idx = device_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, smax = [], set(), None
+        try:
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 8:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    smax = float(f[1])
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            top = sorted(sm)[len(sm) // 2:]          # the busier half of the samples = under load
+            out.update(sm_mhz=statistics.median(top), sm_max_mhz=smax, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle on a bounded sample
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_step(cfg, rows=32, seed=2004):
+    """One bounded sample of the workload on the host: the first layer's forward product for the
+    first `rows` tokens (quantize those rows of X, quantize all of W, dequantize-then-matmul)."""
+    from oracle import binding as ob
+    name, K, N = cfg["linears"][0]
+    X = synth.normal((rows, K), 1.0, seed, device="cpu").float().numpy()
+    W = synth.normal((N, K), 0.02, seed + 1, device="cpu").float().numpy()
+    t0 = time.perf_counter()
+    gx, gw = ob.tensor_amax_scale(X), ob.tensor_amax_scale(W)
+    xc, xs = ob.quantize(X, g=gx)
+    wc, ws = ob.quantize(W, g=gw)
+    ob.gemm(xc, xs, gx, wc, ws, gw, want_T=False)
+    dt = time.perf_counter() - t0
+    flops = 2.0 * rows * K * N
+    return flops, dt, f"layer '{name}' forward product on the first {rows} of {cfg['tokens']} tokens " \
+                      f"(quantize X rows + all of W, dequantize-then-matmul in double)"
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import binding as ob
+    cfg = synth.LLAMA_7B
+    for _ in range(max(args.warmup, 0) and 1):
+        oracle_sample_step(cfg)
+    flops = secs = 0.0
+    sample = ""
+    for _ in range(args.steps):
+        f, dt, sample = oracle_sample_step(cfg)
+        flops += f
+        secs += dt
+    val = flops / secs / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "nvfp4 (e2m1 x ue4m3), f64 accumulate",
+        "data": "synthetic", "config": {"workload": "llama7b_block_linears_fwd_bwd", "tokens": cfg["tokens"],
+                                        "hidden": cfg["hidden"], "sample": sample},
+        "cpu_baseline": {"value": val, "unit": "TFLOPS", "cores": ob.host_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "TFLOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# the GPU arm
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b", choices=["llama7b", "llama350m"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-quantizer", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    from paper_2505_19115_b200 import binding as nb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+    nb.lib()                                      # fails loudly when the CUDA library is missing
+
+    cfg = synth.LLAMA_7B if args.workload == "llama7b" else synth.LLAMA_350M
+    M = cfg["tokens"]
+    peaks, peak_kind = load_peaks()
+
+    # ---- resident inputs: every rank has its own block (replicas; no data-path collective) ----
+    layers = []
+    for li, (name, K, N) in enumerate(cfg["linears"]):
+        X, W, dY = synth.linear_inputs(M, K, N, seed=4000 + 10 * li + 100 * rank, device=dev)
+        layers.append(dict(name=name, K=K, N=N, X=X, W=W, dY=dY,
+                           Y=torch.empty((M, N), dtype=torch.float32, device=dev),
+                           dX=torch.empty((M, K), dtype=torch.float32, device=dev),
+                           dW=torch.empty((N, K), dtype=torch.float32, device=dev)))
+    ws_bytes = max(nb.nvfp4_linear_workspace_bytes(M, l["N"], l["K"], w) for l in layers for w in (0, 1, 2))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    rt = nb.Rounding(nb.RTN)
+    sr = [nb.Rounding(nb.SR, 0, o) for o in range(3)]      # distinct offsets per SR site
+    in_bytes = sum(t.numel() * t.element_size() for l in layers for t in (l["X"], l["W"], l["dY"]))
+
+    def step():
+        for l in layers:
+            nb.nvfp4_linear_fwd(l["X"], l["W"], nb.G_AMAX, rx=rt, rw=rt, out=l["Y"], workspace=ws)
+            nb.nvfp4_linear_bwd_dx(l["dY"], l["W"], nb.G_AMAX, rdy=sr[0], rw=rt, out=l["dX"], workspace=ws)
+            nb.nvfp4_linear_bwd_dw(l["dY"], l["X"], nb.G_AMAX, rdy=sr[1], rx=sr[2], out=l["dW"], workspace=ws)
+
+    launches_per_step = len(layers) * 3 * 7       # 2 x (amax + finalize) + 2 quantize + 1 GEMM per product
+    flops_per_step = block_flops(cfg)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    err_word = nb.nvfp4_device_error_word()
+    if err_word:
+        raise RuntimeError(f"device error word {err_word:#x}: a kernel gave up on a bounded wait")
+    value = flops_per_step * args.steps * world / (ms * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel (the GEMM): same workload, decomposed into the C-ABI's
+    #      quantize and gemm calls so that CUDA events bracket every GEMM launch ----
+    def decomposed_ops(l):
+        ops = []
+        for kind, a, b, ta, tb, ra, rb, out in (("fwd", l["X"], l["W"], False, False, rt, rt, l["Y"]),
+                                                 ("dx", l["dY"], l["W"], False, True, sr[0], rt, l["dX"]),
+                                                 ("dw", l["dY"], l["X"], True, True, sr[1], sr[2], l["dW"])):
+            ops.append((a, b, ta, tb, ra, rb, out))
+        return ops
+
+    gemm_events = []
+    gemm_flops = 0.0
+    roof_steps = min(args.steps, 3)
+    for it in range(roof_steps + 1):
+        for l in layers:
+            for a, b, ta, tb, ra, rb, out in decomposed_ops(l):
+                ga, gb = nb.nvfp4_tensor_amax_scale(a), nb.nvfp4_tensor_amax_scale(b)
+                ac, asf = nb.nvfp4_quantize(a, ta, ga, ra, nb.SF_SWIZZLED)
+                bc, bsf = nb.nvfp4_quantize(b, tb, gb, rb, nb.SF_SWIZZLED)
+                s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                s0.record()
+                nb.nvfp4_gemm(ac, asf, ga, bc, bsf, gb, out=out)
+                s1.record()
+                if it > 0:                       # first pass is warm-up
+                    gemm_events.append((s0, s1))
+                    gemm_flops += 2.0 * out.shape[0] * out.shape[1] * ac.shape[1] * 2
+                del ac, asf, bc, bsf
+    torch.cuda.synchronize()
+    gemm_ms = sum(a.elapsed_time(b) for a, b in gemm_events)
+    n_gemm = len(gemm_events)
+    gemm_tflops = gemm_flops / (gemm_ms * 1e-3) / 1e12
+    clocks = sampler.stop() if rank == 0 else None
+    fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
+    roofline = {
+        "bound": "tensor", "kernel": "gemm_nvfp4_kernel", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
+        "frac": gemm_tflops / fp4_peak, "traffic": GEMM_TRAFFIC_BYTES,
+        "peak_basis": f"{peak_kind} sustained bf16 {peaks['bf16_tflops_sustained']} TFLOP/s x {FP4_OVER_BF16:g} "
+                      f"(nominal dense NVFP4/bf16 ratio); burst basis {peaks['bf16_tflops'] * FP4_OVER_BF16:.0f}; nominal 9000",
+        "launches": n_gemm, "avg_launch_ms": gemm_ms / n_gemm, "flops_per_launch_avg": gemm_flops / n_gemm,
+        "frac_of_nominal_9pf": gemm_tflops / 9000.0,
+    }
+
+    # ---- quantizer bandwidth at 2^28 elements (heavy-tailed inputs), bytes = 2 + 0.5 + 1/16 per element ----
+    quant = None
+    if not args.no_quantizer and rank == 0:
+        for l in layers:
+            l["Y"] = l["dX"] = l["dW"] = None
+        torch.cuda.empty_cache()
+        n_el = 2 ** 28
+        xq = synth.heavy_tailed(synth.square_shape(n_el), seed=1002, device=dev)
+        gq = nb.nvfp4_tensor_amax_scale(xq)
+        codes = torch.empty((xq.shape[0], xq.shape[1] // 2), dtype=torch.uint8, device=dev)
+        sfs = torch.empty(nb.nvfp4_sf_bytes(xq.shape[0], xq.shape[1], nb.SF_SWIZZLED), dtype=torch.uint8, device=dev)
+        quant = {"elements": n_el, "bytes_per_element": 2.5625, "peak_hbm_gbs": peaks["hbm_gbs"], "peak_kind": peak_kind}
+        for label, tr, rr in (("row_rtn", False, rt), ("row_sr", False, nb.Rounding(nb.SR, 1, 0)),
+                              ("transposed_rtn", True, rt), ("transposed_sr", True, nb.Rounding(nb.SR, 1, 0))):
+            for _ in range(3):
+                nb.nvfp4_quantize(xq, tr, gq, rr, nb.SF_SWIZZLED, codes=codes, scales=sfs)
+            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = 10
+            q0.record()
+            for _ in range(reps):
+                nb.nvfp4_quantize(xq, tr, gq, rr, nb.SF_SWIZZLED, codes=codes, scales=sfs)
+            q1.record()
+            torch.cuda.synchronize()
+            gbs = n_el * 2.5625 * reps / (q0.elapsed_time(q1) * 1e-3) / 1e9
+            quant[label] = {"GB/s": gbs, "frac_of_measured_copy": gbs / peaks["hbm_gbs"], "frac_of_8TBs": gbs / 8000.0}
+        del xq, codes, sfs
+        torch.cuda.empty_cache()
+
+    # ---- end to end through the C ABI with host buffers (H2D of every input, D2H of every output) ----
+    e2e = None
+    if not args.no_e2e:
+        for l in layers:
+            for k in ("Y", "dX", "dW"):
+                if l[k] is None:
+                    shape = {"Y": (M, l["N"]), "dX": (M, l["K"]), "dW": (l["N"], l["K"])}[k]
+                    l[k] = torch.empty(shape, dtype=torch.float32, device=dev)
+        host_in = [{k: l[k].cpu().pin_memory() for k in ("X", "W", "dY")} for l in layers]
+        max_out = {k: max(l[k].numel() for l in layers) for k in ("Y", "dX", "dW")}
+        host_out = {k: torch.empty(n, dtype=torch.float32).pin_memory() for k, n in max_out.items()}
+        h2d = sum(t.numel() * t.element_size() for h in host_in for t in h.values())
+        d2h = sum(l[k].numel() * 4 for l in layers for k in ("Y", "dX", "dW"))
+
+        def e2e_step():
+            for l, h in zip(layers, host_in):
+                for k in ("X", "W", "dY"):
+                    l[k].copy_(h[k], non_blocking=True)
+                nb.nvfp4_linear_fwd(l["X"], l["W"], nb.G_AMAX, rx=rt, rw=rt, out=l["Y"], workspace=ws)
+                nb.nvfp4_linear_bwd_dx(l["dY"], l["W"], nb.G_AMAX, rdy=sr[0], rw=rt, out=l["dX"], workspace=ws)
+                nb.nvfp4_linear_bwd_dw(l["dY"], l["X"], nb.G_AMAX, rdy=sr[1], rx=sr[2], out=l["dW"], workspace=ws)
+                for k in ("Y", "dX", "dW"):
+                    host_out[k][:l[k].numel()].copy_(l[k].view(-1), non_blocking=True)
+
+        e2e_steps = max(1, min(args.steps, 3))
+        e2e_step()
+        barrier()
+        f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        f0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        f1.record()
+        barrier()
+        ems = f0.elapsed_time(f1)
+        if dist is not None:
+            t = torch.tensor([ems], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        e2e = {"value": flops_per_step * e2e_steps * world / (ems * 1e-3) / 1e12, "unit": "TFLOPS",
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "ms_per_step": ems / e2e_steps}
+        del host_in, host_out
+
+    # ---- the oracle on the host cores, bounded sample ----
+    cpu = None
+    if rank == 0 and not args.no_cpu and world == 1:
+        from oracle import binding as ob
+        f = secs = 0.0
+        sample = ""
+        for _ in range(2):
+            ff, dt, sample = oracle_sample_step(cfg)
+            f += ff
+            secs += dt
+        cpu = {"value": f / secs / 1e12, "unit": "TFLOPS", "cores": ob.host_threads(), "kind": "oracle",
+               "sample": sample + f"; 2 repetitions, {secs:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "nvfp4 (e2m1 x ue4m3 block scales), fp32 accumulate and output",
+            "data": "synthetic",
+            "config": {"workload": "llama7b_block_linears_fwd_bwd" if args.workload == "llama7b" else "llama350m_block_linears_fwd_bwd",
+                       "tokens": M, "hidden": cfg["hidden"], "linears": [[n, k, o] for n, k, o in cfg["linears"]],
+                       "products_per_step": 15, "rounding": "RtN forward, Philox SR backward/update",
+                       "per_tensor_scale": "amax/(6*448), computed inside every call",
+                       "l2": f"inputs exceed L2: {in_bytes / 2 ** 20:.0f} MiB of operands per step, fp32 outputs on top",
+                       "parallelism": "replicas only (one GPU per rank, no data-path collective)"},
+            "pct_of_fp4_peak": {"of_nominal_9pf": value / world / 9000.0 * 100,
+                                f"of_{peak_kind}_sustained_x4": value / world / fp4_peak * 100},
+            "roofline": roofline, "quantizer": quant, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
