@@ -157,6 +157,35 @@ NVFP4_API int nvfp4_linear_bwd_dw(const void* dY, const void* X, int dtype, int6
                         const nvfp4_rounding* rdy, const nvfp4_rounding* rx,
                         void* dW, int dw_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/*
+ * nvfp4_linear_fwd without a caller-supplied workspace and without any device-memory
+ * allocation (the paper has no counterpart; this is a library convenience).
+ *
+ * It is meant for callers that cannot obtain scratch memory at the call site: a host
+ * program whose framework reserved the whole device for its own memory pool at start-up
+ * (so a cudaMalloc would fail, or would have to be carved out of that pool through an API
+ * the caller does not control), or a latency-critical section in which the implicit
+ * device-wide synchronisation of cudaMalloc/cudaFree is not acceptable.
+ *
+ * The scratch lives in a fixed array of NVFP4_STATIC_WORKSPACE_BYTES in the library's device
+ * image; every GPU on which the library's kernels are loaded holds that much memory until the
+ * process exits.  Arguments and results are those of nvfp4_linear_fwd (X, W, Y are still the
+ * caller's buffers).  A layer whose nvfp4_linear_workspace_bytes(M, N, K, NVFP4_LINEAR_FWD)
+ * exceeds NVFP4_STATIC_WORKSPACE_BYTES is rejected with NVFP4_ERR_WORKSPACE before any launch.
+ *
+ * The first call on each device looks up the array's device address (once per device, with
+ * that device current); make that first call outside any stream capture.  Every call on a
+ * device uses the same array and finds the previous call's contents in it; each call rewrites
+ * all bytes it later reads, so nothing needs clearing by the caller, but two calls that can
+ * overlap on the GPU (different streams, or different host threads) race on it: serialise them.
+ * No cudaMalloc, cudaFree or allocating library routine is called.
+ */
+#define NVFP4_STATIC_WORKSPACE_BYTES (8u << 20)
+NVFP4_API int nvfp4_linear_fwd_static(const void* X, const void* W, int dtype, int64_t M, int64_t N, int64_t K,
+                                      int gscale_mode, const float* gx, const float* gw,
+                                      const nvfp4_rounding* rx, const nvfp4_rounding* rw,
+                                      void* Y, int y_dtype, void* cuda_stream);
+
 /* Reads and clears the device-side error word of the current device (host
  * out-pointer; synchronises the device).  Non-zero means a kernel gave up on a
  * bounded wait and its output is invalid; bits 0-7 identify the wait site. */

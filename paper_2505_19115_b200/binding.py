@@ -65,6 +65,8 @@ def lib():
     for name in ("nvfp4_linear_fwd", "nvfp4_linear_bwd_dx", "nvfp4_linear_bwd_dw"):
         getattr(L, name).restype = ci
         getattr(L, name).argtypes = lin
+    L.nvfp4_linear_fwd_static.restype = ci
+    L.nvfp4_linear_fwd_static.argtypes = [vp, vp, ci, i64, i64, i64, ci, vp, vp, rp, rp, vp, ci, vp]
     L.nvfp4_device_error_word.restype = ci
     L.nvfp4_device_error_word.argtypes = [C.POINTER(C.c_uint32)]
     _lib = L
@@ -189,6 +191,26 @@ def nvfp4_linear_bwd_dw(dY, X, gscale_mode=G_AMAX, gdy=None, gx=None, rdy=None, 
     (M, N), K = dY.shape, X.shape[1]
     return _linear("nvfp4_linear_bwd_dw", LINEAR_BWD_DW, dY, X, M, N, K, (N, K), gscale_mode, gdy, gx,
                    rdy or Rounding(SR, 0, 1), rx or Rounding(SR, 0, 2), out, out_dtype, workspace, stream)
+
+
+STATIC_WORKSPACE_BYTES = 8 << 20
+
+
+def nvfp4_linear_fwd_static(X, W, gscale_mode=G_AMAX, gx=None, gw=None, rx=None, rw=None, out=None,
+                            out_dtype=torch.float32, stream=None):
+    """nvfp4_linear_fwd for callers that cannot allocate or pass scratch memory (for instance when
+    the whole device already belongs to the host framework's pool): the scratch is a fixed
+    STATIC_WORKSPACE_BYTES array inside the library, shared by all calls on a device, so calls
+    that may overlap on the GPU must be serialised.  Larger layers raise (status 5)."""
+    (M, K), N = X.shape, W.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=X.device)
+    rx, rw = rx or Rounding(RTN), rw or Rounding(RTN)
+    assert X.is_contiguous() and W.is_contiguous() and out.is_contiguous() and X.dtype == W.dtype
+    st = lib().nvfp4_linear_fwd_static(_ptr(X), _ptr(W), _dtype_code(X), M, N, K, gscale_mode, _ptr(gx), _ptr(gw),
+                                       C.byref(rx), C.byref(rw), _ptr(out), _dtype_code(out), _stream(stream))
+    _check(st, "nvfp4_linear_fwd_static")
+    return out
 
 
 def nvfp4_device_error_word() -> int:

@@ -115,3 +115,48 @@ extern "C" int nvfp4_linear_bwd_dw(const void* dY, const void* X, int dtype, int
   return run_linear(NVFP4_LINEAR_BWD_DW, dY, X, dtype, M, N, K, gscale_mode, gdy, gx, rdy, rx, dW, dw_dtype,
                     workspace, workspace_bytes, cuda_stream);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Forward product with the scratch in a fixed device array (no allocation anywhere on the path).
+// For callers that cannot get scratch memory when they call: the device may already be fully
+// reserved by the host framework's own pool, or the section may not tolerate the device-wide
+// synchronisation that cudaMalloc / cudaFree imply.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+// Lives in the device image of this library: each GPU that loads it holds these bytes until exit.
+static __device__ __align__(256) unsigned char g_static_workspace[NVFP4_STATIC_WORKSPACE_BYTES];
+
+// In host code `g_static_workspace` is only a handle for the runtime, not a device address; the
+// address a kernel may use comes from cudaGetSymbolAddress, looked up once per device with that
+// device current.
+int static_workspace_address(void** out) {
+  static void* address[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NVFP4_ERR_CUDA;
+  if (!address[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return NVFP4_ERR_CUDA;
+    address[dev] = p;
+  }
+  *out = address[dev];
+  return NVFP4_OK;
+}
+
+}  // namespace
+
+extern "C" int nvfp4_linear_fwd_static(const void* X, const void* W, int dtype, int64_t M, int64_t N, int64_t K,
+                                       int gscale_mode, const float* gx, const float* gw,
+                                       const nvfp4_rounding* rx, const nvfp4_rounding* rw,
+                                       void* Y, int y_dtype, void* cuda_stream) {
+  const size_t need = nvfp4_linear_workspace_bytes(M, N, K, NVFP4_LINEAR_FWD);
+  if (need == 0) return NVFP4_ERR_SHAPE;
+  if (need > (size_t)NVFP4_STATIC_WORKSPACE_BYTES) return NVFP4_ERR_WORKSPACE;  // layer too large for the fixed array
+  if (int st = check_arch()) return st;
+  void* scratch = nullptr;
+  if (int st = static_workspace_address(&scratch)) return st;
+  // The quantizers rewrite every code and scale byte (padding included) that the GEMM reads and
+  // the amax pass clears its own accumulator, so the previous call's contents need no clearing.
+  return run_linear(NVFP4_LINEAR_FWD, X, W, dtype, M, N, K, gscale_mode, gx, gw, rx, rw, Y, y_dtype, scratch,
+                    (size_t)NVFP4_STATIC_WORKSPACE_BYTES, cuda_stream);
+}
