@@ -118,8 +118,10 @@ NVFP4_API int nvfp4_gemm(const uint8_t* a_codes, const uint8_t* a_sf, const floa
                int64_t M, int64_t N, int64_t K,
                void* d, int d_dtype, int64_t ldd, void* cuda_stream);
 
-/* Tuning/testing hook: force the GEMM tile width (128 or 256 output columns per
- * CTA tile); 0 restores the automatic choice.  Process-wide, not thread-safe. */
+/* Tuning/testing hook: force the GEMM kernel variant.  0 restores the automatic
+ * choice; 128 / 256 select the single-CTA kernel with a 128 x {128,256} tile;
+ * 2128 / 2192 / 2256 select the CTA-pair kernel with a 256 x {128,192,256} tile.
+ * Process-wide, not thread-safe. */
 NVFP4_API int nvfp4_gemm_set_tile_n(int bn);
 
 /* Scratch bytes nvfp4_linear_* needs for a layer of shape (M, N, K);

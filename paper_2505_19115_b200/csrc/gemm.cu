@@ -155,6 +155,64 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- cluster / CTA-pair helpers (cta_group::2 path) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory offset in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Tiled copy whose completion bytes are signalled on a barrier that may live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+               ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// Arrives on the barrier at the same offset in both CTAs of the pair once all prior MMAs finish.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_cp_sf_pair(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_nvf4_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\t"
+               "setp.ne.b32 p, %4, 0;\n\t"
+               "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+               : "memory");
+}
+
 // Shared-memory matrix descriptors (64-bit): start address, leading/stride byte offsets (all >> 4),
 // descriptor version 1 at bit 46, swizzle mode at bits 61-63.
 // Operand tiles: K-major, 128-byte swizzle, rows 128 bytes apart, 8-row groups 1024 bytes apart.
@@ -356,6 +414,230 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   }
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// CTA-pair kernel (cta_group::2): a cluster of two CTAs computes a 256 x BN tile.  Each CTA stages
+// its own 128 rows of A, half of the B tile and the scale tiles it needs (its A rows, all BN B
+// rows); the leader CTA issues the MMAs for both, every CTA drains its own 128 accumulator rows.
+// All loads are plain tiled copies (no multicast); the peer's copies signal the leader's barrier.
+// The epilogue goes through shared memory (128-byte swizzle) and leaves as tiled bulk stores.
+// ------------------------------------------------------------------------------------------------
+template <int BN>
+struct Cfg2 {
+  static constexpr int kSfbTiles = (BN % 128 == 0) ? BN / 128 : BN / 128 + 1;
+  static constexpr int kStages = (BN == 128) ? 6 : 5;
+  static constexpr int kAccStages = (BN == 256) ? 1 : 2;
+  static constexpr int kABytes = 128 * BK_BYTES;
+  static constexpr int kBBytes = (BN / 2) * BK_BYTES;
+  static constexpr int kSfaBytes = 2048;
+  static constexpr int kSfbBytes = kSfbTiles * 2048;
+  static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
+  static constexpr int kEpiWarpBytes = 2 * 4096;                   // two 32-row x 128-byte buffers per warp
+  static constexpr int kEpiBytes = 4 * kEpiWarpBytes;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 + 256;
+  static constexpr uint32_t kSfaCol = kAccStages * BN;
+  static constexpr uint32_t kSfCols = 16 + kSfbTiles * 16;
+  static_assert(kStageBytes % 1024 == 0, "stage must keep the 1024-byte swizzle alignment");
+  static_assert(kSfaCol + 2 * kSfCols <= kTmemCols, "tensor memory overflow");
+  static_assert(kSmemBytes <= 232448, "shared memory overflow");
+};
+
+struct Gemm2Params {
+  const float* a_g;
+  const float* b_g;
+  int M, N, K;
+  int tiles_m, tiles_n, k_stages, k_tiles;
+  int a_row_tiles, b_row_tiles;
+};
+
+template <int BN, bool BF16_OUT>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                   const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
+                   const __grid_constant__ CUtensorMap map_d, const Gemm2Params p) {
+  using C = Cfg2<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t epi_base = smem_base + C::kStages * C::kStageBytes;
+  const uint32_t bar_base = epi_base + C::kEpiBytes;
+  uint8_t* bar_gen = smem_gen + C::kStages * C::kStageBytes + C::kEpiBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + C::kAccStages + a); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * C::kStages + 2 * C::kAccStages));
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < C::kAccStages; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
+    *abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 1) tmem_alloc_pair(smem_u32((const void*)tmem_slot), kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                               // both CTAs' barriers exist before any remote signal
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------- TMA producer (both CTAs) -------------------------------
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      constexpr uint32_t kTxPerCta = C::kABytes + C::kBBytes + C::kSfaBytes + C::kSfbBytes;
+      for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+        const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+        const int m0 = tm * 256 + (int)rank * 128, n0 = tn * BN;
+        const int a_rt = min(tm * 2 + (int)rank, p.a_row_tiles - 1);
+        for (int ks = 0; ks < p.k_stages; ++ks) {
+          if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 0x11))) break;
+          const uint32_t st = smem_base + s * C::kStageBytes;
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2u * kTxPerCta);
+          const uint32_t lead_full = map_to_cta(full_bar(s), 0);
+          tma_load_2d_pair(st, &map_a, lead_full, ks * BK_BYTES, m0);
+          tma_load_2d_pair(st + C::kABytes, &map_b, lead_full, ks * BK_BYTES, n0 + (int)rank * (BN / 2));
+          tma_load_2d_pair(st + C::kABytes + C::kBBytes, &map_sfa, lead_full, 0, a_rt * p.k_tiles + ks * 4);
+#pragma unroll
+          for (int h = 0; h < C::kSfbTiles; ++h) {
+            const int rt = min(n0 / 128 + h, p.b_row_tiles - 1);          // rows past N are never stored
+            tma_load_2d_pair(st + C::kABytes + C::kBBytes + C::kSfaBytes + h * 2048, &map_sfb, lead_full, 0,
+                             rt * p.k_tiles + ks * 4);
+          }
+          if (++s == C::kStages) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) {                                    // give copies in flight a bounded time to land
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) {}
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer (leader CTA only) -------------------------------
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = instr_desc(256, BN);
+      int s = 0;
+      uint32_t ph = 0;
+      int acc = 0;
+      uint32_t acc_ph = 0, sfbuf = 0;
+      bool ok = true;
+      for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+        const int tn = tile / p.tiles_m;
+        const uint32_t sfb_off = (uint32_t)((tn * BN) % 128) / 32;         // first scale column of this N tile
+        if (!(ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, 0x12))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int ks = 0; ks < p.k_stages; ++ks) {
+          if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, 0x13))) break;
+          tc_fence_after();
+          const uint32_t st = smem_base + s * C::kStageBytes;
+          const int nkt = min(4, p.k_tiles - ks * 4);
+          const uint32_t sfa_t = tmem_base + C::kSfaCol + sfbuf * C::kSfCols;
+          const uint32_t sfb_t = sfa_t + 16;
+          for (int j = 0; j < nkt; ++j) {
+            tc_cp_sf_pair(sfa_t + 4 * j, sf_desc(st + C::kABytes + C::kBBytes + 512 * j));
+#pragma unroll
+            for (int h = 0; h < C::kSfbTiles; ++h)
+              tc_cp_sf_pair(sfb_t + 4 * C::kSfbTiles * j + 4 * h,
+                            sf_desc(st + C::kABytes + C::kBBytes + C::kSfaBytes + h * 2048 + 512 * j));
+          }
+          const uint64_t adesc = operand_desc(st), bdesc = operand_desc(st + C::kABytes);
+          for (int j = 0; j < nkt; ++j)
+            tc_mma_nvf4_pair(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, sfa_t + 4 * j,
+                             sfb_t + 4 * C::kSfbTiles * j + sfb_off, (ks | j) ? 1u : 0u);
+          tc_commit_pair(empty_bar(s));
+          sfbuf ^= 1u;
+          if (++s == C::kStages) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit_pair(tfull_bar(acc));
+        if (++acc == C::kAccStages) { acc = 0; acc_ph ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------- epilogue (both CTAs) -------------------------------
+    const int quarter = warp & 3;
+    const float alpha = (p.a_g ? __ldg(p.a_g) : 1.0f) * (p.b_g ? __ldg(p.b_g) : 1.0f);
+    const uint32_t my_buf = epi_base + quarter * C::kEpiWarpBytes;
+    constexpr int kChunkCols = BF16_OUT ? 64 : 32;
+    const uint32_t lead_tempty0 = map_to_cta(tempty_bar(0), 0);
+    int acc = 0;
+    uint32_t acc_ph = 0, chunk_no = 0;
+    bool ok = true;
+    for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+      const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+      if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, 0x14))) break;
+      tc_fence_after();
+      const int row0 = tm * 256 + (int)rank * 128 + quarter * 32;
+      const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += kChunkCols, ++chunk_no) {
+        const uint32_t buf = my_buf + (chunk_no & 1u) * 4096u;
+        if (chunk_no >= 2) {                        // the store issued two chunks ago has read this buffer
+          if (lane == 0) tma_store_wait_read<1>();
+          __syncwarp();
+        }
+        uint32_t w[32];
+        if constexpr (BF16_OUT) {
+          uint32_t r0[32], r1[32];
+          tmem_ld32(t_row + c0, r0);
+          tmem_ld32(t_row + c0 + 32, r1);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r0[2 * e]) * alpha, __uint_as_float(r0[2 * e + 1]) * alpha);
+            const __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r1[2 * e]) * alpha, __uint_as_float(r1[2 * e + 1]) * alpha);
+            w[e] = *reinterpret_cast<const uint32_t*>(&h0);
+            w[16 + e] = *reinterpret_cast<const uint32_t*>(&h1);
+          }
+        } else {
+          tmem_ld32(t_row + c0, w);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 32; ++e) w[e] = __float_as_uint(__uint_as_float(w[e]) * alpha);
+        }
+        if (c0 + kChunkCols >= BN) {                // accumulator fully read: hand it back to the leader
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(lead_tempty0 + 8u * acc);
+        }
+        // row = lane: 128 bytes as eight 16-byte pieces, piece index XOR (row & 7) (128-byte swizzle)
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint32_t dst = buf + lane * 128 + ((c ^ (lane & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(w[4 * c]), "r"(w[4 * c + 1]),
+                       "r"(w[4 * c + 2]), "r"(w[4 * c + 3]) : "memory");
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&map_d, buf, tn * BN + c0, row0);
+          tma_store_commit();
+        }
+      }
+      if (++acc == C::kAccStages) { acc = 0; acc_ph ^= 1u; }
+    }
+    if (lane == 0) tma_store_wait_all();
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                               // the peer's MMAs and loads are done before anyone frees or exits
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
@@ -385,6 +667,33 @@ bool make_codes_map(CUtensorMap* map, const uint8_t* base, int64_t rows, int64_t
   const cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Scale tiles as a 2-D tensor of 32-bit words: one 512-byte tile per row, boxes of four tiles.
+bool make_sf_map(CUtensorMap* map, const uint8_t* base, int64_t n_tiles) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {128, (cuuint64_t)n_tiles};
+  const cuuint64_t strides[1] = {512};
+  const cuuint32_t box[2] = {128, 4};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint8_t*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Output D[M, N] (row pitch ldd elements) -> boxes of 32 rows x 128 bytes, 128-byte swizzle.
+bool make_out_map(CUtensorMap* map, void* base, int64_t M, int64_t N, int64_t ldd, bool bf16) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t esz = bf16 ? 2 : 4;
+  const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)ldd * esz};
+  const cuuint32_t box[2] = {(cuuint32_t)(128 / esz), 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides,
+            box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -418,16 +727,52 @@ int launch_gemm(const uint8_t* a_codes, const uint8_t* b_codes, GemmParams p, cu
   return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
+template <int BN, bool BF16_OUT>
+int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParams& g, cudaStream_t s) {
+  using C = Cfg2<BN>;
+  CUtensorMap map_a, map_b, map_sfa, map_sfb, map_d;
+  if (!make_codes_map(&map_a, a_codes, g.M, g.K / 2, 128)) return NVFP4_ERR_CUDA;
+  if (!make_codes_map(&map_b, b_codes, g.N, g.K / 2, BN / 2)) return NVFP4_ERR_CUDA;
+  if (!make_sf_map(&map_sfa, g.a_sf, (int64_t)g.a_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
+  if (!make_sf_map(&map_sfb, g.b_sf, (int64_t)g.b_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
+  if (!make_out_map(&map_d, g.d, g.M, g.N, g.ldd, BF16_OUT)) return NVFP4_ERR_CUDA;
+  Gemm2Params p;
+  p.a_g = g.a_g; p.b_g = g.b_g; p.M = g.M; p.N = g.N; p.K = g.K;
+  p.tiles_m = (g.M + 255) / 256;
+  p.tiles_n = (g.N + BN - 1) / BN;
+  p.k_stages = g.k_stages; p.k_tiles = g.k_tiles;
+  p.a_row_tiles = g.a_row_tiles; p.b_row_tiles = g.b_row_tiles;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(gemm2_nvfp4_kernel<BN, BF16_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             C::kSmemBytes) != cudaSuccess)
+      return NVFP4_ERR_CUDA;
+    attr_set = true;
+  }
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int max_pairs = sm_count() / 2;
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  gemm2_nvfp4_kernel<BN, BF16_OUT><<<2 * pairs, kGemmThreads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
+  return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+template <int BN>
+int launch_gemm2_dt(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParams& g, cudaStream_t s) {
+  return g.d_is_bf16 ? launch_gemm2<BN, true>(a_codes, b_codes, g, s) : launch_gemm2<BN, false>(a_codes, b_codes, g, s);
+}
+
 }  // namespace
 
-int gemm_tile_n_override = 0;  // 0 = automatic; 128 or 256 force a tile width (tuning/tests)
+// 0 = automatic.  128 / 256: single-CTA kernel with that tile width.  2128 / 2192 / 2256: CTA-pair
+// kernel with a 256 x {128,192,256} tile.
+int gemm_tile_n_override = 0;
 
 }  // namespace nvfp4
 
 using namespace nvfp4;
 
 extern "C" int nvfp4_gemm_set_tile_n(int bn) {
-  if (bn != 0 && bn != 128 && bn != 256) return NVFP4_ERR_ENUM;
+  if (bn != 0 && bn != 128 && bn != 256 && bn != 2128 && bn != 2192 && bn != 2256) return NVFP4_ERR_ENUM;
   gemm_tile_n_override = bn;
   return NVFP4_OK;
 }
@@ -457,8 +802,14 @@ extern "C" int nvfp4_gemm(const uint8_t* a_codes, const uint8_t* a_sf, const flo
   p.d_is_bf16 = (d_dtype == NVFP4_BF16);
   p.tiles_m = p.tiles_n = 0;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  int bn = gemm_tile_n_override ? gemm_tile_n_override : 128;
-  return bn == 256 ? launch_gemm<256>(a_codes, b_codes, p, s) : launch_gemm<128>(a_codes, b_codes, p, s);
+  const int bn = gemm_tile_n_override ? gemm_tile_n_override : 2192;
+  switch (bn) {
+    case 128: return launch_gemm<128>(a_codes, b_codes, p, s);
+    case 256: return launch_gemm<256>(a_codes, b_codes, p, s);
+    case 2128: return launch_gemm2_dt<128>(a_codes, b_codes, p, s);
+    case 2256: return launch_gemm2_dt<256>(a_codes, b_codes, p, s);
+    default: return launch_gemm2_dt<192>(a_codes, b_codes, p, s);
+  }
 }
 
 extern "C" int nvfp4_device_error_word(uint32_t* host_out) {

@@ -47,7 +47,7 @@ def _check(gpu_ops, ora_ops, out_dtype=torch.float32):
     return got, ref
 
 
-@pytest.fixture(params=[128, 256])
+@pytest.fixture(params=[128, 256, 2128, 2192, 2256])
 def tile_n(request):
     nb.nvfp4_gemm_set_tile_n(request.param)
     yield request.param
