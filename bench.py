@@ -14,9 +14,7 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
-import tempfile
 import time
 
 import torch
@@ -49,54 +47,64 @@ def block_flops(cfg):
 # clocks
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clock, power and the clock-event reasons of one GPU through NVML from a host
+    thread (every 10 ms) while the timed region runs."""
+    REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20),
+               ("sw_power_cap", 0x4))
 
     def __init__(self, device_index):
         self.idx = device_index
-        self.proc = None
-        self.path = None
+        self.thread = None
+        self.stop_flag = False
+        self.sm, self.power, self.mask = [], [], 0
+        self.smax = None
+        self.error = None
+
+    def _run(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.idx
+            if visible:
+                ids = [v.strip() for v in visible.split(",") if v.strip()]
+                if self.idx < len(ids) and ids[self.idx].isdigit():
+                    idx = int(ids[self.idx])
+            h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.smax = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            while not self.stop_flag:
+                self.sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                try:
+                    self.power.append(pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0)
+                    self.mask |= int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
+                except Exception:
+                    pass
+                time.sleep(0.01)
+        except Exception as e:  # the number is still reported, without a clock record
+            self.error = repr(e)
 
     def start(self):
-        try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            os.close(fd)
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
-        except Exception:
-            self.proc = None
+        import threading
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
+
+    def mark(self):
+        """Drops what was sampled so far (warm-up), so the record covers the timed region only."""
+        self.sm, self.power, self.mask = [], [], 0
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
+        out = {"sm_mhz": None, "sm_max_mhz": self.smax, "reasons": [], "samples": 0}
+        if self.thread is None:
             return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, reasons, smax = [], set(), None
-        try:
-            for line in open(self.path):
-                f = [t.strip() for t in line.split(",")]
-                if len(f) < 8:
-                    continue
-                try:
-                    sm.append(float(f[0]))
-                    smax = float(f[1])
-                except ValueError:
-                    continue
-                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[4:8]):
-                    if v.lower().startswith("active"):
-                        reasons.add(name)
-            os.unlink(self.path)
-        except Exception:
-            pass
-        if sm:
-            top = sorted(sm)[len(sm) // 2:]          # the busier half of the samples = under load
-            out.update(sm_mhz=statistics.median(top), sm_max_mhz=smax, reasons=sorted(reasons), samples=len(sm))
+        self.stop_flag = True
+        self.thread.join(timeout=5)
+        if self.sm:
+            out.update(sm_mhz=statistics.median(self.sm), sm_min_mhz=min(self.sm), sm_max_mhz=self.smax,
+                       reasons=[n for n, bit in self.REASONS if self.mask & bit], samples=len(self.sm))
+            if self.power:
+                out["power_w_max"] = max(self.power)
+        if self.error:
+            out["error"] = self.error
         return out
 
 
@@ -155,7 +163,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama7b", choices=["llama7b", "llama350m"])
@@ -215,19 +223,21 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        step()
-    barrier()
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
+    for _ in range(args.warmup):
+        step()
+    barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    sampler.mark()
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     barrier()
+    clocks = sampler.stop() if rank == 0 else None
     ms = e0.elapsed_time(e1)
     if dist is not None:
         t = torch.tensor([ms], device=dev)
@@ -269,7 +279,6 @@ def main():
     gemm_ms = sum(a.elapsed_time(b) for a, b in gemm_events)
     n_gemm = len(gemm_events)
     gemm_tflops = gemm_flops / (gemm_ms * 1e-3) / 1e12
-    clocks = sampler.stop() if rank == 0 else None
     fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
     roofline = {
         "bound": "tensor", "kernel": "gemm_nvfp4_kernel", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",

@@ -88,23 +88,79 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   return t;
 }
 
-// Bounded wait.  Returns false (and records `site`) if the barrier did not flip within the time
+// Bounded waits.  They return false (and record `site`) if the barrier did not flip within the time
 // limit or another role of this CTA already gave up.
+//
+// mbar_wait spins without pause: for the MMA issuer, whose latency is the kernel's critical path.
+// mbar_wait_relaxed sleeps between polls: every other role waits most of the time, and a dozen
+// warps polling shared memory back to back slow the issuer's own barrier reads several times over.
+__device__ __forceinline__ bool mbar_wait_timeout(uint32_t site, volatile uint32_t* abort_flag, unsigned long long t0) {
+  if (*abort_flag) return true;
+  if (global_timer_ns() - t0 > kWaitLimitNs) {
+    *abort_flag = 1u;
+    atomicOr(&g_error_word, 0x100u | site);
+    return true;
+  }
+  return false;
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
-  for (int i = 0; i < 2048; ++i)
+  for (int i = 0; i < 4096; ++i)
     if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer_ns();
   while (true) {
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (global_timer_ns() - t0 > kWaitLimitNs) {
-      *abort_flag = 1u;
-      atomicOr(&g_error_word, 0x100u | site);
-      return false;
-    }
-    __nanosleep(128);
+    if (mbar_wait_timeout(site, abort_flag, t0)) return false;
   }
+}
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  while (true) {
+    for (int i = 0; i < 256; ++i) {
+      __nanosleep(32);
+      if (mbar_try_wait(bar, parity)) return true;
+    }
+    if (mbar_wait_timeout(site, abort_flag, t0)) return false;
+  }
+}
+// Wait of the MMA-issuing warp.  The poll is a relaxed one: with MMAs in flight an acquiring
+// try_wait stalls its thread for ~170 cycles even when the phase is already complete, a relaxed one
+// for ~40, and the issuer has only 512 cycles per stage.  Nothing the issuer does afterwards reads
+// memory through the generic proxy: it issues tcgen05.mma, whose shared-memory operands were written
+// by the bulk copies that completed the phase, and whose tensor-memory scales are ordered by
+// tcgen05.fence::after_thread_sync.
+__device__ __forceinline__ bool mbar_try_wait_relaxed(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n\t.reg .pred p;\n\t"
+               "mbarrier.try_wait.parity.relaxed.cta.shared::cta.b64 p, [%1], %2;\n\t"
+               "selp.u32 %0, 1, 0, p;\n\t}"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_issuer(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
+  for (int i = 0; i < 4096; ++i)
+    if (mbar_try_wait_relaxed(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  while (true) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait_relaxed(bar, parity)) return true;
+    if (mbar_wait_timeout(site, abort_flag, t0)) return false;
+  }
+}
+// One lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+// Whole-warp wait: lane 0 polls, then every lane observes the completed phase once itself.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
+  bool ok = true;
+  if ((threadIdx.x & 31) == 0) ok = mbar_wait_relaxed(bar, parity, abort_flag, site);
+  ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
+  if (ok) (void)mbar_try_wait(bar, parity);
+  return ok;
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
@@ -153,7 +209,24 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// tcgen05.ld fills its registers asynchronously until tcgen05.wait::ld; this empty statement, placed
+// after the wait, makes every later use of the registers depend on it, so the compiler cannot move
+// such a use above the wait.
+__device__ __forceinline__ void tmem_ld_pin(uint32_t (&r)[32]) {
+#pragma unroll
+  for (int i = 0; i < 32; i += 8)
+    asm volatile("" : "+r"(r[i]), "+r"(r[i + 1]), "+r"(r[i + 2]), "+r"(r[i + 3]), "+r"(r[i + 4]), "+r"(r[i + 5]),
+                      "+r"(r[i + 6]), "+r"(r[i + 7]) :: "memory");
+}
 
 // ---- cluster / CTA-pair helpers (cta_group::2 path) ----
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -167,8 +240,11 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
 }
+// Arrive on a barrier that may live in the peer CTA.  Default semantics (release at CTA scope): a
+// cluster-scope release costs about a thousand cycles here, and the data these arrivals publish
+// lives in tensor memory, whose ordering comes from tcgen05.wait / tcgen05.fence, not from this fence.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -201,9 +277,6 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(bar), "h"((uint16_t)3) : "memory");
 }
-__device__ __forceinline__ void tc_cp_sf_pair(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-}
 __device__ __forceinline__ void tc_mma_nvf4_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
                                                  uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
   asm volatile("{\n\t.reg .pred p;\n\t"
@@ -228,6 +301,18 @@ __device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
 // scales, N >> 3 at bit 17, M >> 4 at bit 24.
 __host__ __device__ constexpr uint32_t instr_desc(int m, int n) {
   return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (0u << 23) | ((uint32_t)(m >> 4) << 24);
+}
+
+// Tile order: panels of kPanel row tiles, column-major inside a panel, so that the CTAs running at
+// the same time share both their A row tiles and their B row tiles (each operand tile is then read
+// by ~8 CTAs instead of one B tile by all of them, and the wave's working set stays small in L2).
+constexpr int kPanel = 8;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
+  const int per_panel = kPanel * tiles_n;
+  const int panel = tile / per_panel, in_panel = tile - panel * per_panel;
+  const int height = min(kPanel, tiles_m - panel * kPanel);
+  tn = in_panel / height;
+  tm = panel * kPanel + in_panel - tn * height;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -276,9 +361,10 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       uint32_t armed = 0, armed_ph = 0;  // per stage: armed at least once / phase of the last arming
       bool ok = true;
       for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-        const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
+        int tm, tn;
+        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
         for (int ks = 0; ks < p.k_stages; ++ks) {
-          if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 1))) break;
+          if (!(ok = mbar_wait_relaxed(empty_bar(s), ph ^ 1u, abort_flag, 1))) break;
           const int kt0 = ks * 4;
           const int nkt = min(4, p.k_tiles - kt0);                        // scale tiles in this stage
           const uint32_t sf_bytes = (uint32_t)nkt * 512u;
@@ -356,8 +442,9 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     uint32_t acc_ph = 0;
     bool ok = true;
     for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-      const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-      if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, 4))) break;
+      int tm, tn;
+        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      if (!(ok = mbar_wait_warp(tfull_bar(acc), acc_ph, abort_flag, 4))) break;
       tc_fence_after();
       const int row = tm * BM + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + acc * C::kAccCols + ((uint32_t)(quarter * 32) << 16);
@@ -366,6 +453,7 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         uint32_t r[32];
         tmem_ld32(t_row + c0, r);
         tmem_ld_wait();
+        tmem_ld_pin(r);
         const int col = tn * BN + c0;
         if (row < p.M && col < p.N) {
           if (p.d_is_bf16) {
@@ -419,9 +507,20 @@ gemm_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 // CTA-pair kernel (cta_group::2): a cluster of two CTAs computes a 256 x BN tile.  Each CTA stages
 // its own 128 rows of A, half of the B tile and the scale tiles it needs (its A rows, all BN B
 // rows); the leader CTA issues the MMAs for both, every CTA drains its own 128 accumulator rows.
-// All loads are plain tiled copies (no multicast); the peer's copies signal the leader's barrier.
+// All loads are plain tiled copies (no multicast); the peer's operand copies signal the leader's
+// barrier.
+//
+// Scales reach tensor memory through registers: four warps per CTA read the stage's scale tiles
+// from shared memory and write them with tcgen05.st into one of several scale buffers, ahead of
+// the MMA issuer.  (A tcgen05.cp per 512-byte scale tile costs 75-120 cycles and an NVFP4 stage
+// needs 12 of them for 512 cycles of MMA work, which caps the kernel near a third of the MMA rate;
+// the register path keeps up with the tensor cores.)
+//
 // The epilogue goes through shared memory (128-byte swizzle) and leaves as tiled bulk stores.
+// Warps: 0 operand producer, 1 MMA issuer, 2-5 epilogue, 6-9 scale movers, 10 scale producer.
 // ------------------------------------------------------------------------------------------------
+constexpr int kGemm2Threads = 352;
+
 template <int BN>
 struct Cfg2 {
   static constexpr int kSfbTiles = (BN % 128 == 0) ? BN / 128 : BN / 128 + 1;
@@ -434,12 +533,19 @@ struct Cfg2 {
   static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
   static constexpr int kEpiWarpBytes = 2 * 4096;                   // two 32-row x 128-byte buffers per warp
   static constexpr int kEpiBytes = 4 * kEpiWarpBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 + 256;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*align*/ + 512 /*barriers*/;
+  // tensor memory: accumulators, then kSfBufs scale buffers of (16 columns for A, 16 per B tile)
   static constexpr uint32_t kSfaCol = kAccStages * BN;
   static constexpr uint32_t kSfCols = 16 + kSfbTiles * 16;
+  static constexpr int kSfBufsFit = (int)((kTmemCols - kSfaCol) / kSfCols);
+  static constexpr int kSfBufs = kSfBufsFit > kStages ? kStages : kSfBufsFit;
+  // with as many scale buffers as stages, buffer b is stage s and needs no barrier of its own
+  static constexpr bool kSfFollowsStage = (kSfBufs == kStages);
+  static constexpr int kNumBarriers = 3 * kStages + 2 * kSfBufs + 2 * kAccStages;
   static_assert(kStageBytes % 1024 == 0, "stage must keep the 1024-byte swizzle alignment");
-  static_assert(kSfaCol + 2 * kSfCols <= kTmemCols, "tensor memory overflow");
+  static_assert(kSfBufs >= 2, "need at least two scale buffers in tensor memory");
   static_assert(kSmemBytes <= 232448, "shared memory overflow");
+  static_assert(8 * kNumBarriers + 8 <= 512, "barrier area overflow");
 };
 
 struct Gemm2Params {
@@ -451,7 +557,7 @@ struct Gemm2Params {
 };
 
 template <int BN, bool BF16_OUT>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemm2Threads, 1)
 gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
                    const __grid_constant__ CUtensorMap map_d, const Gemm2Params p) {
@@ -462,20 +568,27 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   const uint32_t epi_base = smem_base + C::kStages * C::kStageBytes;
   const uint32_t bar_base = epi_base + C::kEpiBytes;
   uint8_t* bar_gen = smem_gen + C::kStages * C::kStageBytes + C::kEpiBytes;
+  // full: operands of both CTAs landed (leader's copy is the one waited on)
+  // sfl:  this CTA's scale tiles landed        empty: the stage's MMAs are done (both CTAs)
+  // sfr:  scale buffer written in both CTAs (leader's copy)   sfe: scale buffer free again (both CTAs)
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
-  auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + a); };
-  auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * C::kStages + C::kAccStages + a); };
-  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * (2 * C::kStages + 2 * C::kAccStages));
+  auto sfl_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (2 * C::kStages + s); };
+  auto sfr_bar = [&](int b) { return bar_base + 8u * (3 * C::kStages + b); };
+  auto sfe_bar = [&](int b) { return bar_base + 8u * (3 * C::kStages + C::kSfBufs + b); };
+  auto tfull_bar = [&](int a) { return bar_base + 8u * (3 * C::kStages + 2 * C::kSfBufs + a); };
+  auto tempty_bar = [&](int a) { return bar_base + 8u * (3 * C::kStages + 2 * C::kSfBufs + C::kAccStages + a); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * C::kNumBarriers);
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const int num_tiles = p.tiles_m * p.tiles_n;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(sfl_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < C::kSfBufs; ++b) { mbar_init(sfr_bar(b), 8); mbar_init(sfe_bar(b), 1); }
     for (int a = 0; a < C::kAccStages; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
     *abort_flag = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -488,127 +601,211 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // The producer and issuer warps run their loops with all 32 lanes (so that loop state, addresses and
+  // descriptors stay warp-uniform) and predicate only the asynchronous instructions on one lane.
   if (warp == 0) {
-    // ------------------------------- TMA producer (both CTAs) -------------------------------
-    if (lane == 0) {
-      int s = 0;
-      uint32_t ph = 0;
-      bool ok = true;
-      constexpr uint32_t kTxPerCta = C::kABytes + C::kBBytes + C::kSfaBytes + C::kSfbBytes;
-      for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-        const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-        const int m0 = tm * 256 + (int)rank * 128, n0 = tn * BN;
-        const int a_rt = min(tm * 2 + (int)rank, p.a_row_tiles - 1);
-        for (int ks = 0; ks < p.k_stages; ++ks) {
-          if (!(ok = mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, 0x11))) break;
-          const uint32_t st = smem_base + s * C::kStageBytes;
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2u * kTxPerCta);
-          const uint32_t lead_full = map_to_cta(full_bar(s), 0);
+    // ------------------------------- operand producer (both CTAs) -------------------------------
+    // One warp can issue a tiled copy every ~75 cycles, so operands and scales have a producer each.
+    const bool issuer = elect_one();
+    int s = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    constexpr uint32_t kOperandTx = C::kABytes + C::kBBytes;       // per CTA, signalled on the leader's barrier
+    for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+      int tm, tn;
+      tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      const int m0 = tm * 256 + (int)rank * 128, n0 = tn * BN + (int)rank * (BN / 2);
+      for (int ks = 0; ks < p.k_stages; ++ks) {
+        if (!(ok = mbar_wait_relaxed(empty_bar(s), ph ^ 1u, abort_flag, 0x11))) break;
+        const uint32_t st = smem_base + s * C::kStageBytes;
+        const uint32_t lead_full = map_to_cta(full_bar(s), 0);
+        if (issuer) {
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2u * kOperandTx);
           tma_load_2d_pair(st, &map_a, lead_full, ks * BK_BYTES, m0);
-          tma_load_2d_pair(st + C::kABytes, &map_b, lead_full, ks * BK_BYTES, n0 + (int)rank * (BN / 2));
-          tma_load_2d_pair(st + C::kABytes + C::kBBytes, &map_sfa, lead_full, 0, a_rt * p.k_tiles + ks * 4);
-#pragma unroll
-          for (int h = 0; h < C::kSfbTiles; ++h) {
-            const int rt = min(n0 / 128 + h, p.b_row_tiles - 1);          // rows past N are never stored
-            tma_load_2d_pair(st + C::kABytes + C::kBBytes + C::kSfaBytes + h * 2048, &map_sfb, lead_full, 0,
-                             rt * p.k_tiles + ks * 4);
-          }
-          if (++s == C::kStages) { s = 0; ph ^= 1u; }
+          tma_load_2d_pair(st + C::kABytes, &map_b, lead_full, ks * BK_BYTES, n0);
         }
+        if (++s == C::kStages) { s = 0; ph ^= 1u; }
       }
-      if (!ok) {                                    // give copies in flight a bounded time to land
-        const unsigned long long t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 200000ull) {}
+    }
+    if (!ok && issuer) {                            // give copies in flight a bounded time to land
+      const unsigned long long t0 = global_timer_ns();
+      while (global_timer_ns() - t0 < 200000ull) {}
+    }
+  } else if (warp == 10) {
+    // ------------------------------- scale producer (both CTAs) -------------------------------
+    const bool issuer = elect_one();
+    int s = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    constexpr uint32_t kScaleTx = C::kSfaBytes + C::kSfbBytes;     // signalled on this CTA's own barrier
+    for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+      int tm, tn;
+      tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      const int a_row = min(tm * 2 + (int)rank, p.a_row_tiles - 1) * p.k_tiles;
+      int b_row[C::kSfbTiles];
+#pragma unroll
+      for (int h = 0; h < C::kSfbTiles; ++h)                       // rows past N are never stored
+        b_row[h] = min((tn * BN) / 128 + h, p.b_row_tiles - 1) * p.k_tiles;
+      for (int ks = 0; ks < p.k_stages; ++ks) {
+        if (!(ok = mbar_wait_relaxed(empty_bar(s), ph ^ 1u, abort_flag, 0x18))) break;
+        const uint32_t sf = smem_base + s * C::kStageBytes + C::kABytes + C::kBBytes;
+        if (issuer) {
+          mbar_arrive_expect_tx(sfl_bar(s), kScaleTx);
+          tma_load_2d(sf, &map_sfa, sfl_bar(s), 0, a_row + ks * 4);
+#pragma unroll
+          for (int h = 0; h < C::kSfbTiles; ++h)
+            tma_load_2d(sf + C::kSfaBytes + h * 2048, &map_sfb, sfl_bar(s), 0, b_row[h] + ks * 4);
+        }
+        if (++s == C::kStages) { s = 0; ph ^= 1u; }
       }
+    }
+    if (!ok && issuer) {
+      const unsigned long long t0 = global_timer_ns();
+      while (global_timer_ns() - t0 < 200000ull) {}
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer (leader CTA only) -------------------------------
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
+      const bool issuer = elect_one();
       constexpr uint32_t idesc = instr_desc(256, BN);
-      int s = 0;
-      uint32_t ph = 0;
-      int acc = 0;
-      uint32_t acc_ph = 0, sfbuf = 0;
+      int s = 0, b = 0, acc = 0;
+      uint32_t ph = 0, bph = 0, acc_ph = 0;
       bool ok = true;
       for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-        const int tn = tile / p.tiles_m;
+        int tm_unused, tn;
+        tile_coords(tile, p.tiles_m, p.tiles_n, tm_unused, tn);
         const uint32_t sfb_off = (uint32_t)((tn * BN) % 128) / 32;         // first scale column of this N tile
-        if (!(ok = mbar_wait(tempty_bar(acc), acc_ph ^ 1u, abort_flag, 0x12))) break;
-        tc_fence_after();
+        if (!(ok = mbar_wait_issuer(tempty_bar(acc), acc_ph ^ 1u, abort_flag, 0x12))) break;
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int ks = 0; ks < p.k_stages; ++ks) {
-          if (!(ok = mbar_wait(full_bar(s), ph, abort_flag, 0x13))) break;
+          if (!(ok = mbar_wait_issuer(full_bar(s), ph, abort_flag, 0x13))) break;
+          if (!(ok = mbar_wait_issuer(sfr_bar(b), bph, abort_flag, 0x15))) break;
           tc_fence_after();
           const uint32_t st = smem_base + s * C::kStageBytes;
           const int nkt = min(4, p.k_tiles - ks * 4);
-          const uint32_t sfa_t = tmem_base + C::kSfaCol + sfbuf * C::kSfCols;
-          const uint32_t sfb_t = sfa_t + 16;
-          for (int j = 0; j < nkt; ++j) {
-            tc_cp_sf_pair(sfa_t + 4 * j, sf_desc(st + C::kABytes + C::kBBytes + 512 * j));
-#pragma unroll
-            for (int h = 0; h < C::kSfbTiles; ++h)
-              tc_cp_sf_pair(sfb_t + 4 * C::kSfbTiles * j + 4 * h,
-                            sf_desc(st + C::kABytes + C::kBBytes + C::kSfaBytes + h * 2048 + 512 * j));
-          }
+          const uint32_t sfa_t = tmem_base + C::kSfaCol + b * C::kSfCols;
+          const uint32_t sfb_t = sfa_t + 16 + sfb_off;
           const uint64_t adesc = operand_desc(st), bdesc = operand_desc(st + C::kABytes);
-          for (int j = 0; j < nkt; ++j)
-            tc_mma_nvf4_pair(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, sfa_t + 4 * j,
-                             sfb_t + 4 * C::kSfbTiles * j + sfb_off, (ks | j) ? 1u : 0u);
-          tc_commit_pair(empty_bar(s));
-          sfbuf ^= 1u;
+          if (issuer) {
+            if (nkt == 4) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                tc_mma_nvf4_pair(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, sfa_t + 4 * j,
+                                 sfb_t + 4 * C::kSfbTiles * j, (ks | j) ? 1u : 0u);
+            } else {
+              for (int j = 0; j < nkt; ++j)
+                tc_mma_nvf4_pair(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, sfa_t + 4 * j,
+                                 sfb_t + 4 * C::kSfbTiles * j, (ks | j) ? 1u : 0u);
+            }
+            tc_commit_pair(empty_bar(s));           // shared-memory stage free in both CTAs
+            if constexpr (!C::kSfFollowsStage) tc_commit_pair(sfe_bar(b));   // scale buffer free in both CTAs
+          }
           if (++s == C::kStages) { s = 0; ph ^= 1u; }
+          if (++b == C::kSfBufs) { b = 0; bph ^= 1u; }
         }
         if (!ok) break;
-        tc_commit_pair(tfull_bar(acc));
+        if (issuer) tc_commit_pair(tfull_bar(acc));
         if (++acc == C::kAccStages) { acc = 0; acc_ph ^= 1u; }
       }
     }
+  } else if (warp >= 6) {                           // warps 6-9 (warp 10 was taken above)
+    // ------------------------------- scale movers (both CTAs) -------------------------------
+    // Shared-memory scale tile: row l (16 bytes) = four 32-row groups x four k-blocks.  Tensor
+    // memory wants exactly that word in lane l of every 32-lane quarter, one column per group.
+    const int quarter = warp & 3;
+    const uint32_t lane_field = (uint32_t)(quarter * 32) << 16;
+    const uint32_t lead_sfr0 = map_to_cta(sfr_bar(0), 0);
+    int s = 0, b = 0;
+    uint32_t ph = 0, bph = 0;
+    bool ok = true;
+    for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+      for (int ks = 0; ks < p.k_stages; ++ks) {
+        if (!(ok = mbar_wait_warp(sfl_bar(s), ph, abort_flag, 0x16))) break;
+        if constexpr (!C::kSfFollowsStage) {        // otherwise buffer b == stage s, free once sfl_bar(s) could be armed
+          if (!(ok = mbar_wait_warp(sfe_bar(b), bph ^ 1u, abort_flag, 0x17))) break;
+        }
+        tc_fence_after();
+        const uint8_t* sf = smem_gen + s * C::kStageBytes + C::kABytes + C::kBBytes + lane * 16;
+        const uint32_t t_sf = tmem_base + C::kSfaCol + b * C::kSfCols + lane_field;
+        {
+          uint32_t r[16];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint4 v = *reinterpret_cast<const uint4*>(sf + j * 512);
+            r[4 * j] = v.x; r[4 * j + 1] = v.y; r[4 * j + 2] = v.z; r[4 * j + 3] = v.w;
+          }
+          tmem_st16(t_sf, r);
+        }
+#pragma unroll
+        for (int c = 0; c < C::kSfbTiles; ++c) {    // 16 columns at a time: column x = 4*T*j + 4*h + w
+          uint32_t r[16];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int x = 16 * c + 4 * q, j = x / (4 * C::kSfbTiles), h = (x / 4) % C::kSfbTiles;
+            const uint4 v = *reinterpret_cast<const uint4*>(sf + C::kSfaBytes + h * 2048 + j * 512);
+            r[4 * q] = v.x; r[4 * q + 1] = v.y; r[4 * q + 2] = v.z; r[4 * q + 3] = v.w;
+          }
+          tmem_st16(t_sf + 16 + 16 * c, r);
+        }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(lead_sfr0 + 8u * b);
+        if (++s == C::kStages) { s = 0; ph ^= 1u; }
+        if (++b == C::kSfBufs) { b = 0; bph ^= 1u; }
+      }
+    }
   } else {
-    // ------------------------------- epilogue (both CTAs) -------------------------------
+    // ------------------------------- epilogue (both CTAs, warps 2-5) -------------------------------
     const int quarter = warp & 3;
     const float alpha = (p.a_g ? __ldg(p.a_g) : 1.0f) * (p.b_g ? __ldg(p.b_g) : 1.0f);
     const uint32_t my_buf = epi_base + quarter * C::kEpiWarpBytes;
     constexpr int kChunkCols = BF16_OUT ? 64 : 32;
+    constexpr int kLoads = kChunkCols / 32;
     const uint32_t lead_tempty0 = map_to_cta(tempty_bar(0), 0);
     int acc = 0;
     uint32_t acc_ph = 0, chunk_no = 0;
     bool ok = true;
     for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-      const int tm = tile % p.tiles_m, tn = tile / p.tiles_m;
-      if (!(ok = mbar_wait(tfull_bar(acc), acc_ph, abort_flag, 0x14))) break;
+      int tm, tn;
+        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      if (!(ok = mbar_wait_warp(tfull_bar(acc), acc_ph, abort_flag, 0x14))) break;
       tc_fence_after();
       const int row0 = tm * 256 + (int)rank * 128 + quarter * 32;
       const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
+      uint32_t r[kLoads][32];
+#pragma unroll
+      for (int l = 0; l < kLoads; ++l) tmem_ld32(t_row + 32 * l, r[l]);
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += kChunkCols, ++chunk_no) {
         const uint32_t buf = my_buf + (chunk_no & 1u) * 4096u;
-        if (chunk_no >= 2) {                        // the store issued two chunks ago has read this buffer
-          if (lane == 0) tma_store_wait_read<1>();
-          __syncwarp();
-        }
+        tmem_ld_wait();
+#pragma unroll
+        for (int l = 0; l < kLoads; ++l) tmem_ld_pin(r[l]);
         uint32_t w[32];
         if constexpr (BF16_OUT) {
-          uint32_t r0[32], r1[32];
-          tmem_ld32(t_row + c0, r0);
-          tmem_ld32(t_row + c0 + 32, r1);
-          tmem_ld_wait();
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r0[2 * e]) * alpha, __uint_as_float(r0[2 * e + 1]) * alpha);
-            const __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r1[2 * e]) * alpha, __uint_as_float(r1[2 * e + 1]) * alpha);
+            const __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[0][2 * e]) * alpha, __uint_as_float(r[0][2 * e + 1]) * alpha);
+            const __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[1][2 * e]) * alpha, __uint_as_float(r[1][2 * e + 1]) * alpha);
             w[e] = *reinterpret_cast<const uint32_t*>(&h0);
             w[16 + e] = *reinterpret_cast<const uint32_t*>(&h1);
           }
         } else {
-          tmem_ld32(t_row + c0, w);
-          tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) w[e] = __float_as_uint(__uint_as_float(w[e]) * alpha);
+          for (int e = 0; e < 32; ++e) w[e] = __float_as_uint(__uint_as_float(r[0][e]) * alpha);
         }
-        if (c0 + kChunkCols >= BN) {                // accumulator fully read: hand it back to the leader
+        if (c0 + kChunkCols < BN) {                 // next chunk's accumulator read overlaps this chunk's store
+#pragma unroll
+          for (int l = 0; l < kLoads; ++l) tmem_ld32(t_row + c0 + kChunkCols + 32 * l, r[l]);
+        } else {                                    // accumulator fully read: hand it back to the leader
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(lead_tempty0 + 8u * acc);
+        }
+        if (chunk_no >= 2) {                        // the store issued two chunks ago has read this buffer
+          if (lane == 0) tma_store_wait_read<1>();
+          __syncwarp();
         }
         // row = lane: 128 bytes as eight 16-byte pieces, piece index XOR (row & 7) (128-byte swizzle)
 #pragma unroll
@@ -752,7 +949,7 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
   const int tiles = p.tiles_m * p.tiles_n;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  gemm2_nvfp4_kernel<BN, BF16_OUT><<<2 * pairs, kGemmThreads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
+  gemm2_nvfp4_kernel<BN, BF16_OUT><<<2 * pairs, kGemm2Threads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
   return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
@@ -802,13 +999,13 @@ extern "C" int nvfp4_gemm(const uint8_t* a_codes, const uint8_t* a_sf, const flo
   p.d_is_bf16 = (d_dtype == NVFP4_BF16);
   p.tiles_m = p.tiles_n = 0;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  const int bn = gemm_tile_n_override ? gemm_tile_n_override : 2192;
+  const int bn = gemm_tile_n_override ? gemm_tile_n_override : 2256;
   switch (bn) {
     case 128: return launch_gemm<128>(a_codes, b_codes, p, s);
     case 256: return launch_gemm<256>(a_codes, b_codes, p, s);
     case 2128: return launch_gemm2_dt<128>(a_codes, b_codes, p, s);
-    case 2256: return launch_gemm2_dt<256>(a_codes, b_codes, p, s);
-    default: return launch_gemm2_dt<192>(a_codes, b_codes, p, s);
+    case 2192: return launch_gemm2_dt<192>(a_codes, b_codes, p, s);
+    default: return launch_gemm2_dt<256>(a_codes, b_codes, p, s);
   }
 }
 
