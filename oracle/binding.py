@@ -13,6 +13,7 @@ from . import build as _build
 _lib = None
 
 _u8p = np.ctypeslib.ndpointer(dtype=np.uint8, flags="C_CONTIGUOUS")
+_u16p = np.ctypeslib.ndpointer(dtype=np.uint16, flags="C_CONTIGUOUS")
 _f32p = np.ctypeslib.ndpointer(dtype=np.float32, flags="C_CONTIGUOUS")
 _i64p = np.ctypeslib.ndpointer(dtype=np.int64, flags="C_CONTIGUOUS")
 _u32p = np.ctypeslib.ndpointer(dtype=np.uint32, flags="C_CONTIGUOUS")
@@ -31,12 +32,14 @@ def lib():
         L.nvfp4o_e4m3_decode.argtypes = [C.c_uint8]
         L.nvfp4o_philox4x32_10.restype = None
         L.nvfp4o_philox4x32_10.argtypes = [_u32p, _u32p, _u32p]
-        L.nvfp4o_block_random_bytes.restype = None
-        L.nvfp4o_block_random_bytes.argtypes = [C.c_uint64, C.c_uint64, C.c_uint64, _u8p]
+        L.nvfp4o_block_random_u16.restype = None
+        L.nvfp4o_block_random_u16.argtypes = [C.c_uint64, C.c_uint64, C.c_uint64, _u16p]
+        L.nvfp4o_word_random_u16.restype = None
+        L.nvfp4o_word_random_u16.argtypes = [C.c_uint32, _u16p]
         L.nvfp4o_round_rtn.restype = C.c_uint8
         L.nvfp4o_round_rtn.argtypes = [C.c_float]
         L.nvfp4o_round_sr.restype = C.c_uint8
-        L.nvfp4o_round_sr.argtypes = [C.c_float, C.c_uint8]
+        L.nvfp4o_round_sr.argtypes = [C.c_float, C.c_uint16]
         q = [_f32p, C.c_int64, C.c_int64, C.c_float, C.c_int, C.c_uint64, C.c_uint64, _u8p, _u8p, C.c_int]
         L.nvfp4o_quantize.restype = None
         L.nvfp4o_quantize.argtypes = q
@@ -92,9 +95,15 @@ def philox4x32_10(key, ctr):
     return out
 
 
-def block_random_bytes(seed: int, offset: int, block: int):
-    out = np.zeros(16, dtype=np.uint8)
-    lib().nvfp4o_block_random_bytes(seed, offset, block, out)
+def block_random_u16(seed: int, offset: int, block: int):
+    out = np.zeros(16, dtype=np.uint16)
+    lib().nvfp4o_block_random_u16(seed, offset, block, out)
+    return out
+
+
+def word_random_u16(word: int):
+    out = np.zeros(4, dtype=np.uint16)
+    lib().nvfp4o_word_random_u16(word, out)
     return out
 
 
@@ -102,8 +111,8 @@ def round_rtn(y: float) -> int:
     return int(lib().nvfp4o_round_rtn(float(np.float32(y))))
 
 
-def round_sr(y: float, u8: int) -> int:
-    return int(lib().nvfp4o_round_sr(float(np.float32(y)), u8))
+def round_sr(y: float, r16: int) -> int:
+    return int(lib().nvfp4o_round_sr(float(np.float32(y)), r16))
 
 
 def quantize(x, g=1.0, mode=RTN, seed=0, offset=0, transposed=False, nthreads=None):

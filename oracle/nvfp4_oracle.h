@@ -38,16 +38,23 @@ float nvfp4o_e4m3_decode(uint8_t code);
 /* Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw 2011). */
 void nvfp4o_philox4x32_10(const uint32_t key[2], const uint32_t ctr[4], uint32_t out[4]);
 
-/* The 16 random bytes of block B: counter (B_lo, B_hi, offset_lo, offset_hi),
- * key (seed_lo, seed_hi); the four output words little-endian give bytes 0..15. */
-void nvfp4o_block_random_bytes(uint64_t seed, uint64_t offset, uint64_t block, uint8_t out[16]);
+/* The four 16-bit random integers that one Philox output word gives to four
+ * consecutive elements: elements 0,1 share bytes 0 (low half) and 2 (high half) of
+ * the word, elements 2,3 share bytes 1 and 3; the odd element of each pair reads
+ * its 16 bits in reversed order. */
+void nvfp4o_word_random_u16(uint32_t w, uint16_t out[4]);
+
+/* The 16 random integers of block B: counter (B_lo, B_hi, offset_lo, offset_hi),
+ * key (seed_lo, seed_hi); output word q serves elements 4q..4q+3. */
+void nvfp4o_block_random_u16(uint64_t seed, uint64_t offset, uint64_t block, uint16_t out[16]);
 
 /* Section 1: RtN maps y in [0,6] to the closest grid magnitude (ties to the
  * code with an even mantissa bit); SR picks one of the two neighbours with
- * probability given by the distance, using one random byte.  Both return the
- * 3-bit magnitude code. */
+ * probability given by the distance, using a 16-bit random integer r: with f the
+ * position of y inside its grid step, it rounds up iff floor(f*2^16) + r >= 2^16.
+ * Both return the 3-bit magnitude code. */
 uint8_t nvfp4o_round_rtn(float y);
-uint8_t nvfp4o_round_sr(float y, uint8_t u8);
+uint8_t nvfp4o_round_sr(float y, uint16_t r16);
 
 /* Quantize a logical [Rq, Kq] fp32 tensor (row stride Kq) in blocks of 16 along
  * Kq.  mode 0 = RtN, 1 = SR.  codes: Rq*Kq/2 bytes (element 2i in the low

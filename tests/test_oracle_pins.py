@@ -100,16 +100,38 @@ def test_philox_known_answers():
         assert [int(o) for o in out] == v[6:10]
 
 
-def test_block_random_bytes_are_little_endian_words_of_the_counter():
+def _rev16(v):
+    return int(f"{v:016b}"[::-1], 2)
+
+
+def test_word_random_integers_use_every_bit_twice_and_pairs_mirror_each_other():
+    # one-hot words: bit b of bytes 0/2 reaches elements 0 and 1 only, of bytes 1/3 elements 2 and 3
+    # only; the even element takes the byte pair as (low, high), the odd one the same 16 bits mirrored
+    for bit in range(32):
+        byte, k = divmod(bit, 8)
+        r = [int(v) for v in ob.word_random_u16(1 << bit)]
+        pos = k + (8 if byte >= 2 else 0)
+        if byte in (0, 2):
+            assert r == [1 << pos, 1 << (15 - pos), 0, 0]
+        else:
+            assert r == [0, 0, 1 << pos, 1 << (15 - pos)]
+    rng = np.random.default_rng(5)
+    for w in rng.integers(0, 2 ** 32, 200):
+        r = [int(v) for v in ob.word_random_u16(int(w))]
+        assert r[1] == _rev16(r[0]) and r[3] == _rev16(r[2])
+        assert r[0] | (r[2] << 16) == (w & 0xFF) | ((w >> 16 & 0xFF) << 8) | ((w >> 8 & 0xFF) << 16) | ((w >> 24) << 24)
+
+
+def test_block_random_integers_come_from_the_words_of_the_counter():
     seed, offset, block = 0x0123456789ABCDEF, 0x1122334455667788, 0xA1B2C3D4E5F60718
     words = ob.philox4x32_10([seed & 0xFFFFFFFF, seed >> 32],
                              [block & 0xFFFFFFFF, block >> 32, offset & 0xFFFFFFFF, offset >> 32])
-    want = np.frombuffer(words.astype("<u4").tobytes(), dtype=np.uint8)
-    assert np.array_equal(ob.block_random_bytes(seed, offset, block), want)
-    # different block / offset / seed -> different bytes
-    assert not np.array_equal(ob.block_random_bytes(seed, offset, block + 1), want)
-    assert not np.array_equal(ob.block_random_bytes(seed, offset + 1, block), want)
-    assert not np.array_equal(ob.block_random_bytes(seed + 1, offset, block), want)
+    want = np.concatenate([ob.word_random_u16(int(w)) for w in words])
+    assert np.array_equal(ob.block_random_u16(seed, offset, block), want)
+    # different block / offset / seed -> different integers
+    assert not np.array_equal(ob.block_random_u16(seed, offset, block + 1), want)
+    assert not np.array_equal(ob.block_random_u16(seed, offset + 1, block), want)
+    assert not np.array_equal(ob.block_random_u16(seed + 1, offset, block), want)
 
 
 # ---------------------------------------------------------------- rounding
@@ -140,27 +162,39 @@ def _sr_neighbours(y):
     return lo, hi
 
 
-def test_sr_exact_distribution_over_all_bytes():
-    rng = np.random.default_rng(2)
-    ys = np.concatenate([rng.uniform(0, 6, 300), np.array(GRID), [0.001, 5.999, 1.999, 2.001, 3.999, 4.001]])
-    for y in ys.astype(np.float32):
+def test_sr_exact_distribution_over_all_random_integers():
+    # all 2^16 random integers for a few values: support, exact count of round-ups, monotonicity
+    for y in np.array([0.3, 1.26, 2.9, 4.000001, 5.999, 0.0001], dtype=np.float32):
         lo, hi = _sr_neighbours(float(y))
-        vals = np.array([GRID[ob.round_sr(float(y), u)] for u in range(256)])
-        assert set(vals.tolist()) <= {lo, hi}
-        if lo == hi:                                         # representable values never move
-            assert np.all(vals == lo)
-            continue
         delta = hi - lo
         f = (Fraction(float(y)) - Fraction(lo)) / Fraction(delta)
-        ups = sum(1 for u in range(256) if Fraction(2 * u + 1, 512) < f)
+        ups = int(f * 65536)                                  # floor
+        vals = np.array([GRID[ob.round_sr(float(y), r)] for r in range(65536)])
+        assert set(vals.tolist()) <= {lo, hi}
         assert int(np.sum(vals == hi)) == ups
-        # rounding up happens for the smallest bytes (monotone in u)
-        assert np.all(np.diff((vals == hi).astype(int)) <= 0)
-        assert abs(vals.mean() - float(y)) <= delta / 512 + 1e-12
+        assert np.all(np.diff((vals == hi).astype(int)) >= 0)  # the largest integers round up
+        assert 0 <= float(y) - vals.mean() <= delta / 65536 + 1e-12
+
+
+def test_sr_threshold_for_many_values():
+    rng = np.random.default_rng(2)
+    ys = np.concatenate([rng.uniform(0, 6, 2000), np.array(GRID), [0.001, 5.999, 1.999, 2.001, 3.999, 4.001, 1e-6]])
+    for y in ys.astype(np.float32):
+        lo, hi = _sr_neighbours(float(y))
+        if lo == hi:                                          # representable values never move
+            assert all(GRID[ob.round_sr(float(y), r)] == lo for r in (0, 1, 32768, 65535))
+            continue
+        f = (Fraction(float(y)) - Fraction(lo)) / Fraction(hi - lo)
+        F = int(f * 65536)
+        assert GRID[ob.round_sr(float(y), 0)] == lo
+        assert GRID[ob.round_sr(float(y), 65535 - F)] == lo
+        if F > 0:
+            assert GRID[ob.round_sr(float(y), 65536 - F)] == hi
+            assert GRID[ob.round_sr(float(y), 65535)] == hi
 
 
 def test_sr_unbiased_over_seeded_draws():
-    # 10^4 Philox-seeded draws of the same block: mean within 3 sigma (+ the 8-bit bias bound)
+    # 10^4 Philox-seeded draws of the same block: mean within 3 sigma (+ the 16-bit truncation bound)
     x = np.array([[0.3, -0.7, 1.1, 1.6, 2.2, -2.9, 3.3, 4.7, 5.5, 0.05, 6.0, -0.26, 0.9, 1.9, 3.9, -5.9]],
                  dtype=np.float32)
     n = 10000
@@ -176,15 +210,29 @@ def test_sr_unbiased_over_seeded_draws():
     var = np.maximum(acc2 / n - mean ** 2, 0)
     for j in range(16):
         lo, hi = _sr_neighbours(abs(float(x[0, j])))
-        bound = 3 * np.sqrt(var[j] / n) + (hi - lo) / 512 + 1e-9
+        bound = 3 * np.sqrt(var[j] / n) + (hi - lo) / 65536 + 1e-9
         assert abs(mean[j] - float(x[0, j])) <= bound, (j, mean[j], x[0, j], bound)
+
+
+def test_sr_neighbouring_elements_round_independently_enough():
+    # elements 0/1 (and 2/3) of a word share their 16 random bits in mirrored order: the joint
+    # frequency of "both round up" must still be the product of the two probabilities
+    y = np.float32(1.25)                                      # f = 1/2 for both
+    rng = np.random.default_rng(9)
+    both = n = 0
+    for w in rng.integers(0, 2 ** 32, 20000):
+        r = ob.word_random_u16(int(w))
+        a, b = ob.round_sr(float(y), int(r[0])) == 3, ob.round_sr(float(y), int(r[1])) == 3
+        both += a and b
+        n += 1
+    assert abs(both / n - 0.25) < 0.015
 
 
 def test_sr_variance_closed_form():
     # y uniform within one grid step: E[err^2] = delta^2/6 under SR, delta^2/12 under RtN
     rng = np.random.default_rng(3)
     ys = rng.uniform(2.0, 3.0, 40000).astype(np.float32)
-    us = rng.integers(0, 256, ys.size)
+    us = rng.integers(0, 65536, ys.size)
     sr = np.array([GRID[ob.round_sr(float(y), int(u))] for y, u in zip(ys, us)])
     rt = np.array([GRID[ob.round_rtn(float(y))] for y in ys])
     assert abs(np.mean((sr - ys) ** 2) - 1 / 6) < 0.01
@@ -302,7 +350,7 @@ def test_quantize_global_scale():
     assert ob.tensor_amax_scale(np.zeros(5, dtype=np.float32)) == 1.0
 
 
-def test_quantize_sr_uses_block_indexed_bytes_and_is_reproducible():
+def test_quantize_sr_uses_block_indexed_integers_and_is_reproducible():
     rng = np.random.default_rng(7)
     x = torch.from_numpy(rng.standard_normal((5, 64)).astype(np.float32)).to(torch.bfloat16).float().numpy()
     c1, s1 = ob.quantize(x, mode=ob.SR, seed=11, offset=3, nthreads=1)
@@ -315,7 +363,7 @@ def test_quantize_sr_uses_block_indexed_bytes_and_is_reproducible():
     # rebuild every code from the per-element rule and the bytes of block r*(K/16)+kb
     for r in range(5):
         for kb in range(4):
-            rnd = ob.block_random_bytes(11, 3, r * 4 + kb)
+            rnd = ob.block_random_u16(11, 3, r * 4 + kb)
             d = np.float32(ob.e4m3_decode(int(s1[r, kb])))
             inv = np.float32(1.0) / d
             for j in range(16):
