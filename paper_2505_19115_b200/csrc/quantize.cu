@@ -23,81 +23,107 @@ struct QuantParams {
   int64_t k_tiles;  // ceil(nkb / 4)
 };
 
-// One block of 16 values -> 8 bytes of codes (lo, hi words) and one scale byte.
-// c = (1/6)/g, g = per-tensor scale.  `blk` is the block's linear index (Philox counter).
+// Reciprocal of every block scale a tensor can have: entry q = 1 / (decode(q) * g), one IEEE
+// division each, 0 for the zero scale.  A block then costs one shared-memory read, not a division.
+__device__ __forceinline__ void build_inv_table(float* inv_table, float g) {
+  for (int q = threadIdx.x; q < 128; q += blockDim.x)
+    inv_table[q] = (q == 0) ? 0.0f : __fdiv_rn(1.0f, __fmul_rn(e4m3_decode((uint32_t)q), g));
+}
+
+// 16 values (signed, already widened to fp32) and their amax -> 8 bytes of codes (lo, hi words)
+// and one scale byte.  c = (1/6)/g.  `blk` is the block's linear index (Philox counter).
 template <bool SR>
-__device__ __forceinline__ void quantize_block(const float (&v)[16], float c, float g,
-                                               const QuantParams& p, uint64_t blk,
-                                               uint32_t& lo, uint32_t& hi, uint32_t& sf) {
-  float amax = 0.0f;
-#pragma unroll
-  for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(v[j]));
+__device__ __forceinline__ void encode_block(const float (&v)[16], float amax, float c, const float* inv_table,
+                                             const QuantParams& p, uint64_t blk,
+                                             uint32_t& lo, uint32_t& hi, uint32_t& sf) {
   const uint32_t q = e4m3_encode(__fmul_rn(amax, c));
-  const float d = __fmul_rn(e4m3_decode(q), g);
-  const float inv = (q == 0u) ? 0.0f : __fdiv_rn(1.0f, d);
+  const float inv = inv_table[q];
   sf = q;
-  uint32_t w[2] = {0u, 0u};
-  if constexpr (!SR) {
+  float y[16];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float y0 = fminf(__fmul_rn(fabsf(v[2 * j]), inv), 6.0f);
-      const float y1 = fminf(__fmul_rn(fabsf(v[2 * j + 1]), inv), 6.0f);
-      uint32_t b = e2m1x2_rn(y0, y1);
-      b |= ((__float_as_uint(v[2 * j]) >> 28) & 0x8u) | ((__float_as_uint(v[2 * j + 1]) >> 24) & 0x80u);
-      w[j >> 2] |= b << (8 * (j & 3));
-    }
+  for (int j = 0; j < 16; ++j) y[j] = __fmul_rn(v[j], inv);     // the sign rides along; the conversions clamp at 6
+  if constexpr (!SR) {
+    lo = e2m1x8_rn(y, 0);
+    hi = e2m1x8_rn(y, 8);
   } else {
     const uint4 r4 = philox4x32_10(p.seed_lo, p.seed_hi, (uint32_t)blk, (uint32_t)(blk >> 32), p.off_lo, p.off_hi);
-    const uint32_t rw[4] = {r4.x, r4.y, r4.z, r4.w};
-#pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const uint32_t u = (rw[j >> 2] >> (8 * (j & 3))) & 0xFFu;
-      const float y = fminf(__fmul_rn(fabsf(v[j]), inv), 6.0f);
-      const uint32_t nib = e2m1_sr(y, u) | ((__float_as_uint(v[j]) >> 28) & 0x8u);
-      w[j >> 3] |= nib << (4 * (j & 7));
+    lo = e2m1x8_rs(y, 0, r4.x, r4.y);
+    hi = e2m1x8_rs(y, 8, r4.z, r4.w);
+  }
+}
+
+// max |.| of two packed bf16 pairs, per half (the sign bits of the result are meaningless)
+__device__ __forceinline__ uint32_t absmax_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
+// One block of 16 contiguous source values.
+template <typename T>
+struct Block16;
+
+template <>
+struct Block16<__nv_bfloat16> {
+  uint32_t w[8];
+  __device__ __forceinline__ void load(const __nv_bfloat16* src, bool aligned32) {
+    if (aligned32) {
+      asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                   : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                   : "l"(src));
+    } else {
+      const uint4 a = __ldg(reinterpret_cast<const uint4*>(src));
+      const uint4 b = __ldg(reinterpret_cast<const uint4*>(src) + 1);
+      w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w; w[4] = b.x; w[5] = b.y; w[6] = b.z; w[7] = b.w;
     }
   }
-  lo = w[0];
-  hi = w[1];
-}
-
-__device__ __forceinline__ void unpack_bf16x8(const uint4& q, float* v) {
-  const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+  __device__ __forceinline__ float unpack(float (&v)[16]) const {
+    uint32_t m = absmax_bf16x2(absmax_bf16x2(absmax_bf16x2(w[0], w[1]), absmax_bf16x2(w[2], w[3])),
+                               absmax_bf16x2(absmax_bf16x2(w[4], w[5]), absmax_bf16x2(w[6], w[7])));
+    m &= 0x7FFF7FFFu;
+    const uint32_t top = max(m >> 16, m & 0xFFFFu);            // non-negative bf16 patterns order as integers
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    v[2 * i] = __uint_as_float(w[i] << 16);
-    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    for (int i = 0; i < 8; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+    return __uint_as_float(top << 16);
   }
-}
+};
 
-template <typename T>
-__device__ __forceinline__ void load_block16(const T* src, float (&v)[16]) {
-  if constexpr (sizeof(T) == 2) {
-    const uint4 a = __ldg(reinterpret_cast<const uint4*>(src));
-    const uint4 b = __ldg(reinterpret_cast<const uint4*>(src) + 1);
-    unpack_bf16x8(a, v);
-    unpack_bf16x8(b, v + 8);
-  } else {
+template <>
+struct Block16<float> {
+  float4 f[4];
+  __device__ __forceinline__ void load(const float* src, bool) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) f[i] = __ldg(reinterpret_cast<const float4*>(src) + i);
+  }
+  __device__ __forceinline__ float unpack(float (&v)[16]) const {
+    float amax = 0.0f;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const float4 f = __ldg(reinterpret_cast<const float4*>(src) + i);
-      v[4 * i] = f.x; v[4 * i + 1] = f.y; v[4 * i + 2] = f.z; v[4 * i + 3] = f.w;
+      v[4 * i] = f[i].x; v[4 * i + 1] = f[i].y; v[4 * i + 2] = f[i].z; v[4 * i + 3] = f[i].w;
     }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) amax = fmaxf(amax, fabsf(v[j]));
+    return amax;
   }
-}
+};
 
 // -------------------------------------------------------------------------------------------------
 // Row quantizer: CTA tile = 128 rows x 32 blocks (512 columns); warp w takes rows w, w+8, ...;
-// lane = block within the row segment, so a warp reads 1 KB (bf16) of one row per step and
-// writes 256 contiguous code bytes.  Swizzled scales are staged in shared memory and leave as
-// eight contiguous 512-byte tiles.
+// lane = block within the row segment, so a warp reads 1 KB (bf16) of one row per step (one
+// 256-bit load per lane when rows are 32-byte aligned) and writes 256 contiguous code bytes.
+// Several rows are in flight per thread, kept packed.  Swizzled scales are staged in shared
+// memory and leave as eight contiguous 512-byte tiles.
 // -------------------------------------------------------------------------------------------------
 constexpr int kRowTileRows = 128;
 constexpr int kSfChunkPitch = 528;  // 512 + 16: spreads the eight k-tiles over different banks
 
 template <typename T, bool SR, bool SWZ>
-__global__ void __launch_bounds__(kThreads) quantize_row_kernel(const QuantParams p) {
+__global__ void __launch_bounds__(kThreads, 3) quantize_row_kernel(const QuantParams p) {
   __shared__ __align__(16) uint8_t sf_s[SWZ ? 8 * kSfChunkPitch : 16];
+  __shared__ float inv_table[128];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t kb = (int64_t)blockIdx.x * 32 + lane;
   const int64_t row0 = (int64_t)blockIdx.y * kRowTileRows;
@@ -105,31 +131,35 @@ __global__ void __launch_bounds__(kThreads) quantize_row_kernel(const QuantParam
   const float g = p.gptr ? __ldg(p.gptr) : 1.0f;
   const float c = __fdiv_rn(__fdiv_rn(1.0f, 6.0f), g);
   const T* x = static_cast<const T*>(p.x);
+  const bool aligned32 = ((reinterpret_cast<uintptr_t>(x) | (uintptr_t)(p.ld * (int64_t)sizeof(T))) & 31u) == 0;
 
+  build_inv_table(inv_table, g);
   if constexpr (SWZ) {
     for (int i = threadIdx.x; i < 8 * kSfChunkPitch / 16; i += kThreads)
       reinterpret_cast<uint4*>(sf_s)[i] = make_uint4(0, 0, 0, 0);
-    __syncthreads();
   }
+  __syncthreads();
 
-  constexpr int U = 4;  // rows in flight per thread
+  constexpr int U = (sizeof(T) == 2) ? 4 : 2;  // rows in flight per thread (32 packed registers)
 #pragma unroll 1
   for (int it = 0; it < kRowTileRows / 8; it += U) {
-    float v[U][16];
+    Block16<T> raw[U];
     bool ok[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int64_t r = row0 + warp + 8 * (it + u);
       ok[u] = kb_ok && r < p.rows;
-      if (ok[u]) load_block16<T>(x + r * p.ld + kb * 16, v[u]);
+      if (ok[u]) raw[u].load(x + r * p.ld + kb * 16, aligned32);
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       if (!ok[u]) continue;
       const int rl = warp + 8 * (it + u);
       const int64_t r = row0 + rl;
+      float v[16];
+      const float amax = raw[u].unpack(v);
       uint32_t lo, hi, sf;
-      quantize_block<SR>(v[u], c, g, p, (uint64_t)(r * p.nkb + kb), lo, hi, sf);
+      encode_block<SR>(v, amax, c, inv_table, p, (uint64_t)(r * p.nkb + kb), lo, hi, sf);
       *reinterpret_cast<uint2*>(p.codes + (r * p.nkb + kb) * 8) = make_uint2(lo, hi);
       if constexpr (SWZ) {
         sf_s[(lane >> 2) * kSfChunkPitch + (rl & 31) * 16 + (rl >> 5) * 4 + (lane & 3)] = (uint8_t)sf;
@@ -173,7 +203,7 @@ struct TTile {
 };
 
 template <typename T, bool SR, bool SWZ>
-__global__ void __launch_bounds__(kThreads) quantize_transposed_kernel(const QuantParams p) {
+__global__ void __launch_bounds__(kThreads, 3) quantize_transposed_kernel(const QuantParams p) {
   using TT = TTile<T>;
   extern __shared__ __align__(16) uint8_t smem[];
   T* tile = reinterpret_cast<T*>(smem);                                        // [kRows][64]
@@ -186,6 +216,8 @@ __global__ void __launch_bounds__(kThreads) quantize_transposed_kernel(const Qua
   const T* x = static_cast<const T*>(p.x);
   const float g = p.gptr ? __ldg(p.gptr) : 1.0f;
   const float c = __fdiv_rn(__fdiv_rn(1.0f, 6.0f), g);
+  __shared__ float inv_table[128];
+  build_inv_table(inv_table, g);                              // published by the barrier after the tile lands
 
   // ---- stage the input tile ----
   constexpr int kElemsPerChunk = 16 / (int)sizeof(T);
@@ -205,31 +237,48 @@ __global__ void __launch_bounds__(kThreads) quantize_transposed_kernel(const Qua
   __syncthreads();
 
   // ---- quantize: lane -> columns (2*lane, 2*lane+1), warp -> row blocks ----
+  // Staging rows are ordered even columns first (column cl -> row (cl & 1) * 32 + cl / 2), so that a
+  // warp's 8-byte code stores and its scale bytes fall into distinct banks.
 #pragma unroll 1
   for (int rb = warp; rb < TT::kRowBlocks; rb += kThreads / 32) {
-    float va[16], vb[16];
+    float va[16], vb[16], amax_a, amax_b;
+    if constexpr (sizeof(T) == 2) {
+      uint32_t w[16];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const T* e = tile + (rb * 16 + j) * kTCols + 2 * lane;
-      if constexpr (sizeof(T) == 2) {
-        const uint32_t w = *reinterpret_cast<const uint32_t*>(e);
-        va[j] = __uint_as_float(w << 16);
-        vb[j] = __uint_as_float(w & 0xFFFF0000u);
-      } else {
-        const float2 f = *reinterpret_cast<const float2*>(e);
+      for (int j = 0; j < 16; ++j) w[j] = *reinterpret_cast<const uint32_t*>(tile + (rb * 16 + j) * kTCols + 2 * lane);
+      uint32_t m[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) m[j] = absmax_bf16x2(w[2 * j], w[2 * j + 1]);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) m[j] = absmax_bf16x2(m[2 * j], m[2 * j + 1]);
+      const uint32_t mm = absmax_bf16x2(absmax_bf16x2(m[0], m[1]), absmax_bf16x2(m[2], m[3])) & 0x7FFF7FFFu;
+      amax_a = __uint_as_float(mm << 16);                     // low halves = column 2*lane
+      amax_b = __uint_as_float(mm & 0xFFFF0000u);             // high halves = column 2*lane + 1
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        va[j] = __uint_as_float(w[j] << 16);
+        vb[j] = __uint_as_float(w[j] & 0xFFFF0000u);
+      }
+    } else {
+      amax_a = amax_b = 0.0f;
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const float2 f = *reinterpret_cast<const float2*>(tile + (rb * 16 + j) * kTCols + 2 * lane);
         va[j] = f.x;
         vb[j] = f.y;
+        amax_a = fmaxf(amax_a, fabsf(f.x));
+        amax_b = fmaxf(amax_b, fabsf(f.y));
       }
     }
     const int64_t kb = r0 / 16 + rb;
     const int64_t ca = c0 + 2 * lane;
     uint32_t lo, hi, sf;
-    quantize_block<SR>(va, c, g, p, (uint64_t)(ca * p.nkb + kb), lo, hi, sf);
-    *reinterpret_cast<uint2*>(code_s + (2 * lane) * TT::kCodePitch + rb * 8) = make_uint2(lo, hi);
-    sf_s[(2 * lane) * TT::kRowBlocks + rb] = (uint8_t)sf;
-    quantize_block<SR>(vb, c, g, p, (uint64_t)((ca + 1) * p.nkb + kb), lo, hi, sf);
-    *reinterpret_cast<uint2*>(code_s + (2 * lane + 1) * TT::kCodePitch + rb * 8) = make_uint2(lo, hi);
-    sf_s[(2 * lane + 1) * TT::kRowBlocks + rb] = (uint8_t)sf;
+    encode_block<SR>(va, amax_a, c, inv_table, p, (uint64_t)(ca * p.nkb + kb), lo, hi, sf);
+    *reinterpret_cast<uint2*>(code_s + lane * TT::kCodePitch + rb * 8) = make_uint2(lo, hi);
+    sf_s[rb * kTCols + lane] = (uint8_t)sf;
+    encode_block<SR>(vb, amax_b, c, inv_table, p, (uint64_t)((ca + 1) * p.nkb + kb), lo, hi, sf);
+    *reinterpret_cast<uint2*>(code_s + (32 + lane) * TT::kCodePitch + rb * 8) = make_uint2(lo, hi);
+    sf_s[rb * kTCols + 32 + lane] = (uint8_t)sf;
   }
   __syncthreads();
 
@@ -240,7 +289,8 @@ __global__ void __launch_bounds__(kThreads) quantize_transposed_kernel(const Qua
     const int id = threadIdx.x + i * kThreads;
     const int cl = id / TT::kRowBlocks, u = id % TT::kRowBlocks;
     if (c0 + cl < p.cols && kb0 + u < p.nkb) {
-      const uint2 val = *reinterpret_cast<const uint2*>(code_s + cl * TT::kCodePitch + u * 8);
+      const int srow = (cl & 1) * 32 + (cl >> 1);
+      const uint2 val = *reinterpret_cast<const uint2*>(code_s + srow * TT::kCodePitch + u * 8);
       *reinterpret_cast<uint2*>(p.codes + ((c0 + cl) * p.nkb + kb0 + u) * 8) = val;
     }
   }
@@ -252,7 +302,10 @@ __global__ void __launch_bounds__(kThreads) quantize_transposed_kernel(const Qua
       const int cl = id / kKt, t = id % kKt;
       const int64_t kt = kb0 / 4 + t;
       if (kt >= p.k_tiles) continue;
-      const uint32_t val = *reinterpret_cast<const uint32_t*>(sf_s + cl * TT::kRowBlocks + t * 4);
+      const int srow = (cl & 1) * 32 + (cl >> 1);
+      const uint8_t* s4 = sf_s + (t * 4) * kTCols + srow;
+      const uint32_t val = (uint32_t)s4[0] | ((uint32_t)s4[kTCols] << 8) | ((uint32_t)s4[2 * kTCols] << 16) |
+                           ((uint32_t)s4[3 * kTCols] << 24);
       *reinterpret_cast<uint32_t*>(p.scales + sf_swizzled_offset(c0 + cl, kt * 4, p.k_tiles)) = val;
       if (fill_upper)
         *reinterpret_cast<uint32_t*>(p.scales + sf_swizzled_offset(c0 + cl + 64, kt * 4, p.k_tiles)) = 0u;
@@ -260,7 +313,8 @@ __global__ void __launch_bounds__(kThreads) quantize_transposed_kernel(const Qua
   } else {
     for (int id = threadIdx.x; id < kTCols * TT::kRowBlocks; id += kThreads) {
       const int cl = id / TT::kRowBlocks, u = id % TT::kRowBlocks;
-      if (c0 + cl < p.cols && kb0 + u < p.nkb) p.scales[(c0 + cl) * p.nkb + kb0 + u] = sf_s[id];
+      const int srow = (cl & 1) * 32 + (cl >> 1);
+      if (c0 + cl < p.cols && kb0 + u < p.nkb) p.scales[(c0 + cl) * p.nkb + kb0 + u] = sf_s[u * kTCols + srow];
     }
   }
 }
@@ -279,10 +333,8 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const T* x, int64_t rows
     const int64_t r = i / vec_per_row, vcol = i % vec_per_row;
     const uint4 q = __ldg(reinterpret_cast<const uint4*>(x + r * ld + vcol * kVec));
     if constexpr (sizeof(T) == 2) {
-      float v[8];
-      unpack_bf16x8(q, v);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(v[j]));
+      const uint32_t m = absmax_bf16x2(absmax_bf16x2(q.x, q.y), absmax_bf16x2(q.z, q.w)) & 0x7FFF7FFFu;
+      amax = fmaxf(amax, fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u)));
     } else {
       amax = fmaxf(fmaxf(fabsf(__uint_as_float(q.x)), fabsf(__uint_as_float(q.y))),
                    fmaxf(fmaxf(fabsf(__uint_as_float(q.z)), fabsf(__uint_as_float(q.w))), amax));
