@@ -97,6 +97,24 @@ NVFP4_API int nvfp4_quantize(const void* x, int dtype, int64_t rows, int64_t col
                    int transposed, const float* global_scale, const nvfp4_rounding* rounding /* host */,
                    uint8_t* codes, uint8_t* scales, int sf_layout, void* cuda_stream);
 
+/*
+ * Both quantizations of one tensor from a single read: Q(x) with blocks along cols (as
+ * nvfp4_quantize with transposed == 0, rounding_row) and Q(x^T) with blocks along rows (as
+ * transposed == 1, rounding_t).  Eq. 4-6 need every operand in both orientations (Q(dY) in Eq. 5 and
+ * Q(dY^T) in Eq. 6, Q(X) in Eq. 4 and Q(X^T) in Eq. 6, Q(W) in Eq. 4 and Q(W^T) in Eq. 5); each
+ * output is bit-identical to what the corresponding nvfp4_quantize call writes.
+ * rows and cols must both be multiples of 16.  codes_row: rows*cols/2 bytes, scales_row:
+ * nvfp4_sf_bytes(rows, cols, sf_layout); codes_t: cols*rows/2 bytes, scales_t:
+ * nvfp4_sf_bytes(cols, rows, sf_layout).  bf16 tensors whose rows and cols are multiples of 32 take
+ * the fused kernel (one read, 3.125 bytes of traffic per element); others run the two
+ * single-output kernels.  Alignment and errors as for nvfp4_quantize.
+ */
+NVFP4_API int nvfp4_quantize_dual(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                        const float* global_scale,
+                        const nvfp4_rounding* rounding_row /* host */, uint8_t* codes_row, uint8_t* scales_row,
+                        const nvfp4_rounding* rounding_t /* host */, uint8_t* codes_t, uint8_t* scales_t,
+                        int sf_layout, void* cuda_stream);
+
 /* Per-tensor scale g = max|x| / (6*448), or 1.0f for an all-zero tensor, written
  * to *global_scale_out (device).  The paper defines only the block scale; this
  * optional factor keeps small-magnitude gradients inside the E4M3 scale range. */

@@ -53,6 +53,8 @@ def lib():
     L.nvfp4_sf_bytes.argtypes = [i64, i64, ci]
     L.nvfp4_quantize.restype = ci
     L.nvfp4_quantize.argtypes = [vp, ci, i64, i64, i64, ci, vp, rp, vp, vp, ci, vp]
+    L.nvfp4_quantize_dual.restype = ci
+    L.nvfp4_quantize_dual.argtypes = [vp, ci, i64, i64, i64, vp, rp, vp, vp, rp, vp, vp, ci, vp]
     L.nvfp4_tensor_amax_scale.restype = ci
     L.nvfp4_tensor_amax_scale.argtypes = [vp, ci, i64, i64, i64, vp, vp]
     L.nvfp4_gemm.restype = ci
@@ -123,6 +125,29 @@ def nvfp4_quantize(x: torch.Tensor, transposed: bool = False, global_scale: torc
                               _stream(stream))
     _check(st, "nvfp4_quantize")
     return codes, scales
+
+
+def nvfp4_quantize_dual(x: torch.Tensor, global_scale: torch.Tensor = None, rounding_row: Rounding = None,
+                        rounding_t: Rounding = None, sf_layout: int = SF_LINEAR, stream=None):
+    """Row and transposed quantization from one read.  Returns (codes_row, scales_row, codes_t, scales_t)."""
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    rounding_row = rounding_row or Rounding()
+    rounding_t = rounding_t or Rounding()
+
+    def bufs(Rq, Kq):
+        codes = torch.empty((Rq, max(Kq // 2, 1)), dtype=torch.uint8, device=x.device)
+        if sf_layout == SF_LINEAR:
+            return codes, torch.empty((Rq, max(Kq // 16, 1)), dtype=torch.uint8, device=x.device)
+        return codes, torch.empty(max(nvfp4_sf_bytes(Rq, Kq, sf_layout), 16), dtype=torch.uint8, device=x.device)
+
+    cr, sr = bufs(rows, cols)
+    ct, stt = bufs(cols, rows)
+    st = lib().nvfp4_quantize_dual(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), _ptr(global_scale),
+                                   C.byref(rounding_row), _ptr(cr), _ptr(sr), C.byref(rounding_t), _ptr(ct), _ptr(stt),
+                                   sf_layout, _stream(stream))
+    _check(st, "nvfp4_quantize_dual")
+    return cr, sr, ct, stt
 
 
 def nvfp4_tensor_amax_scale(x: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:

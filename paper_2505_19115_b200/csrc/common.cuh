@@ -17,6 +17,13 @@ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 // Checks that the current device is a compute-capability 10.x part (cached per device).
 int check_arch();
 
+// Tile quantizer (quantize_tile.cu): transposed output, optionally the row output from the same read.
+bool tile_quantizer_eligible(int dtype, int64_t rows, int64_t cols, bool dual);
+int tile_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, const float* g, bool dual,
+                  const nvfp4_rounding* rt, uint8_t* codes_t, uint8_t* scales_t,
+                  const nvfp4_rounding* rr, uint8_t* codes_r, uint8_t* scales_r, int sf_layout, cudaStream_t s);
+int tile_error_word(unsigned int* out);
+
 // ---------------------------------------------------------------------------------------------
 // Scale-factor layout (128 rows x 4 blocks per 512-byte tile, k-tiles contiguous per row tile)
 // ---------------------------------------------------------------------------------------------

@@ -14,6 +14,7 @@
 #include <cuda_bf16.h>
 
 #include "common.cuh"
+#include "tensor_map.cuh"
 
 namespace nvfp4 {
 namespace {
@@ -838,22 +839,6 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
 // ------------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
 // Packed codes [rows, row_bytes] -> box of (128 bytes x box_rows), 128-byte swizzle, zero fill.
 bool make_codes_map(CUtensorMap* map, const uint8_t* base, int64_t rows, int64_t row_bytes, int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
@@ -1014,6 +999,9 @@ extern "C" int nvfp4_device_error_word(uint32_t* host_out) {
   unsigned int w = 0, zero = 0;
   if (cudaMemcpyFromSymbol(&w, g_error_word, sizeof(w)) != cudaSuccess) return NVFP4_ERR_CUDA;
   if (w != 0 && cudaMemcpyToSymbol(g_error_word, &zero, sizeof(zero)) != cudaSuccess) return NVFP4_ERR_CUDA;
+  unsigned int tile_w = 0;
+  if (int st = tile_error_word(&tile_w)) return st;
+  w |= tile_w;
   *host_out = w;
   return NVFP4_OK;
 }

@@ -1,0 +1,296 @@
+// Tile quantizer for bf16 tensors: one read of x[rows, cols] produces the transposed NVFP4
+// quantization (blocks of 16 along the row axis, output stored [cols, rows/2]) and, optionally, the
+// row quantization (blocks along the column axis) of the same tile.  This is the producer fusion
+// for the operands that Eq. 4-6 need in both orientations: dY as Q(dY) for Eq. 5 and Q(dY^T) for
+// Eq. 6, X as Q(X) for Eq. 4 and Q(X^T) for Eq. 6, W as Q(W) for Eq. 4 and Q(W^T) for Eq. 5.
+//
+// A CTA takes a tile of 256 rows x 64 columns (32 KB).  One thread fetches it with a tiled bulk
+// copy (128-byte swizzle, zero fill outside the tensor); all threads quantize from shared memory;
+// the packed codes are staged in shared memory and leave as tiled bulk stores (which clip at the
+// tensor edge), the scales as plain stores.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "quantize_core.cuh"
+#include "tensor_map.cuh"
+
+namespace nvfp4 {
+namespace {
+
+constexpr int kTileRows = 256;
+constexpr int kTileCols = 64;
+constexpr int kTileBytes = kTileRows * kTileCols * 2;                 // 32 KB, rows of 128 bytes
+constexpr int kCodesTBytes = kTileCols * (kTileRows / 2);             // 64 output rows x 128 bytes
+constexpr int kCodesRBytes = kTileRows * (kTileCols / 2);             // 256 output rows x 32 bytes
+constexpr int kSfTBytes = kTileCols * (kTileRows / 16);               // [16 row blocks][64 columns]
+constexpr int kSfRBytes = 2 * 512;                                    // two scale tiles (128 rows x 4 blocks)
+constexpr int kTileSmem = kTileBytes + kCodesTBytes + kCodesRBytes + kSfTBytes + kSfRBytes + 1024 /*align*/;
+constexpr unsigned long long kTileWaitLimitNs = 2000000000ull;
+
+struct TileParams {
+  const float* gptr;
+  int64_t rows, cols;
+  // transposed output (always): quantized shape (cols, rows)
+  uint32_t t_seed_lo, t_seed_hi, t_off_lo, t_off_hi;
+  uint8_t* t_scales;
+  int64_t t_nkb, t_k_tiles;
+  // row output (DUAL only): quantized shape (rows, cols)
+  uint32_t r_seed_lo, r_seed_hi, r_off_lo, r_off_hi;
+  uint8_t* r_scales;
+  int64_t r_nkb, r_k_tiles;
+};
+
+__device__ unsigned int g_tile_error_word = 0;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// byte offset of (row, byte) inside a tile of 128-byte rows stored with the 128-byte swizzle
+__device__ __forceinline__ uint32_t swz128(uint32_t row, uint32_t byte) {
+  return row * 128u + ((((byte >> 4) ^ (row & 7u)) << 4) | (byte & 15u));
+}
+
+template <bool SR_T, bool DUAL, bool SR_R, bool SWZ>
+__global__ void __launch_bounds__(kThreads, 3)
+quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_ct,
+                     const __grid_constant__ CUtensorMap map_cr, const TileParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((1024u - (smem_addr(smem_raw) & 1023u)) & 1023u);
+  uint8_t* tile = smem;                                   // [256][128 B], swizzled
+  uint8_t* codes_t = tile + kTileBytes;                   // [64][128 B], swizzled
+  uint8_t* codes_r = codes_t + kCodesTBytes;              // [256][32 B]
+  uint8_t* sf_t = codes_r + kCodesRBytes;                 // [16][64]
+  uint8_t* sf_r = sf_t + kSfTBytes;                       // [2][512]
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ float inv_table[128];
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t c0 = (int64_t)blockIdx.x * kTileCols;
+  const int64_t r0 = (int64_t)blockIdx.y * kTileRows;
+  const float g = p.gptr ? __ldg(p.gptr) : 1.0f;
+  const float c = __fdiv_rn(__fdiv_rn(1.0f, 6.0f), g);
+
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bar)));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(&bar)), "r"(kTileBytes) : "memory");
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_addr(tile)), "l"(&map_x), "r"(smem_addr(&bar)), "r"((int)c0), "r"((int)r0) : "memory");
+  }
+  build_inv_table(inv_table, g);
+  __syncthreads();                                        // barrier initialised, table published
+  {
+    // bounded wait for the tile; on a timeout every thread leaves without storing anything
+    const uint32_t b = smem_addr(&bar);
+    uint32_t done = 0;
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 0; !done; ++spin) {
+      asm volatile("{\n\t.reg .pred q;\n\tmbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                   : "=r"(done) : "r"(b) : "memory");
+      if (!done && (spin & 255u) == 255u) {
+        unsigned long long now;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+        if (t0 == 0) t0 = now;
+        if (now - t0 > kTileWaitLimitNs) {
+          if (threadIdx.x == 0) atomicOr(&g_tile_error_word, 0x200u);
+          return;
+        }
+      }
+    }
+  }
+
+  // ---- transposed output: lane -> columns (2*lane, 2*lane+1), warp -> row blocks ----
+  // Codes are staged as [column][128 bytes] with the 128-byte swizzle the tiled store expects.
+  QuantParams qt;
+  qt.seed_lo = p.t_seed_lo; qt.seed_hi = p.t_seed_hi; qt.off_lo = p.t_off_lo; qt.off_hi = p.t_off_hi;
+#pragma unroll 1
+  for (int rb = warp; rb < kTileRows / 16; rb += kThreads / 32) {
+    uint32_t w[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) w[j] = *reinterpret_cast<const uint32_t*>(tile + swz128(rb * 16 + j, 4 * lane));
+    uint32_t m[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) m[j] = absmax_bf16x2(w[2 * j], w[2 * j + 1]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) m[j] = absmax_bf16x2(m[2 * j], m[2 * j + 1]);
+    const uint32_t mm = absmax_bf16x2(absmax_bf16x2(m[0], m[1]), absmax_bf16x2(m[2], m[3])) & 0x7FFF7FFFu;
+    float va[16], vb[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      va[j] = __uint_as_float(w[j] << 16);                    // column 2*lane
+      vb[j] = __uint_as_float(w[j] & 0xFFFF0000u);            // column 2*lane + 1
+    }
+    const int64_t kb = r0 / 16 + rb;
+    const int64_t ca = c0 + 2 * lane;
+    uint32_t lo, hi, sf;
+    encode_block<SR_T>(va, __uint_as_float(mm << 16), c, inv_table, qt, (uint64_t)(ca * p.t_nkb + kb), lo, hi, sf);
+    *reinterpret_cast<uint2*>(codes_t + swz128(2 * lane, rb * 8)) = make_uint2(lo, hi);
+    sf_t[rb * kTileCols + 2 * lane] = (uint8_t)sf;
+    encode_block<SR_T>(vb, __uint_as_float(mm & 0xFFFF0000u), c, inv_table, qt, (uint64_t)((ca + 1) * p.t_nkb + kb), lo, hi, sf);
+    *reinterpret_cast<uint2*>(codes_t + swz128(2 * lane + 1, rb * 8)) = make_uint2(lo, hi);
+    sf_t[rb * kTileCols + 2 * lane + 1] = (uint8_t)sf;
+  }
+
+  // ---- row output: thread -> (row, block of 16 columns); four rows per thread ----
+  if constexpr (DUAL) {
+    QuantParams qr;
+    qr.seed_lo = p.r_seed_lo; qr.seed_hi = p.r_seed_hi; qr.off_lo = p.r_off_lo; qr.off_hi = p.r_off_hi;
+    const int kbl = threadIdx.x & 3;                          // block within the tile's 64 columns
+#pragma unroll 1
+    for (int i = 0; i < kTileRows / 64; ++i) {
+      const int rl = i * 64 + (threadIdx.x >> 2);
+      const uint4 a = *reinterpret_cast<const uint4*>(tile + swz128(rl, kbl * 32));
+      const uint4 b = *reinterpret_cast<const uint4*>(tile + swz128(rl, kbl * 32 + 16));
+      Block16<__nv_bfloat16> blk;
+      blk.w[0] = a.x; blk.w[1] = a.y; blk.w[2] = a.z; blk.w[3] = a.w;
+      blk.w[4] = b.x; blk.w[5] = b.y; blk.w[6] = b.z; blk.w[7] = b.w;
+      float v[16];
+      const float amax = blk.unpack(v);
+      uint32_t lo, hi, sf;
+      encode_block<SR_R>(v, amax, c, inv_table, qr, (uint64_t)((r0 + rl) * p.r_nkb + c0 / 16 + kbl), lo, hi, sf);
+      *reinterpret_cast<uint2*>(codes_r + rl * 32 + kbl * 8) = make_uint2(lo, hi);
+      if constexpr (SWZ) {
+        sf_r[(rl >> 7) * 512 + (rl & 31) * 16 + ((rl >> 5) & 3) * 4 + kbl] = (uint8_t)sf;
+      } else {
+        if (r0 + rl < p.rows && c0 / 16 + kbl < p.r_nkb) p.r_scales[(r0 + rl) * p.r_nkb + c0 / 16 + kbl] = (uint8_t)sf;
+      }
+    }
+  }
+
+  // ---- codes out: tiled bulk stores from the staging buffers (clipped at the tensor edge) ----
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(&map_ct), "r"(smem_addr(codes_t)), "r"((int)(r0 / 2)), "r"((int)c0) : "memory");
+    if constexpr (DUAL)
+      asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                   ::"l"(&map_cr), "r"(smem_addr(codes_r)), "r"((int)(c0 / 2)), "r"((int)r0) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  }
+
+  // ---- scales out ----
+  const int64_t kb0 = r0 / 16;
+  if constexpr (SWZ) {
+    // transposed scales: one 32-bit word = four row blocks of one column
+    const bool fill_upper = ((c0 & 127) == 0) && (c0 + kTileCols >= p.cols);   // nobody else owns rows 64..127
+    for (int id = threadIdx.x; id < kTileCols * 4; id += kThreads) {
+      const int cl = id >> 2, t = id & 3;
+      const int64_t kt = kb0 / 4 + t;
+      if (kt >= p.t_k_tiles) continue;
+      const uint8_t* s4 = sf_t + (t * 4) * kTileCols + cl;
+      const uint32_t val = (uint32_t)s4[0] | ((uint32_t)s4[kTileCols] << 8) | ((uint32_t)s4[2 * kTileCols] << 16) |
+                           ((uint32_t)s4[3 * kTileCols] << 24);
+      *reinterpret_cast<uint32_t*>(p.t_scales + sf_swizzled_offset(c0 + cl, kt * 4, p.t_k_tiles)) = val;
+      if (fill_upper)
+        *reinterpret_cast<uint32_t*>(p.t_scales + sf_swizzled_offset(c0 + cl + 64, kt * 4, p.t_k_tiles)) = 0u;
+    }
+    if constexpr (DUAL) {
+      // row scales: the tile owns two whole 512-byte scale tiles (128 rows x this k-tile)
+      if (threadIdx.x < 64) {
+        const int h = threadIdx.x >> 5, i = threadIdx.x & 31;
+        if (r0 + h * 128 < p.rows) {
+          const uint4 val = *reinterpret_cast<const uint4*>(sf_r + h * 512 + i * 16);
+          *reinterpret_cast<uint4*>(p.r_scales + ((r0 / 128 + h) * p.r_k_tiles + c0 / 64) * 512 + i * 16) = val;
+        }
+      }
+    }
+  } else {
+    for (int id = threadIdx.x; id < kTileCols * (kTileRows / 16); id += kThreads) {
+      const int cl = id >> 4, u = id & 15;
+      if (c0 + cl < p.cols && kb0 + u < p.t_nkb) p.t_scales[(c0 + cl) * p.t_nkb + kb0 + u] = sf_t[u * kTileCols + cl];
+    }
+  }
+  if (threadIdx.x == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging must outlive the stores' reads
+}
+
+bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* base, uint64_t inner, uint64_t outer,
+                 uint64_t pitch_bytes, uint32_t box_inner, uint32_t box_outer, CUtensorMapSwizzle swz) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {inner, outer};
+  const cuuint64_t strides[1] = {pitch_bytes};
+  const cuuint32_t box[2] = {box_inner, box_outer};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool SR_T, bool DUAL, bool SR_R, bool SWZ>
+cudaError_t launch_tile(const CUtensorMap& mx, const CUtensorMap& mct, const CUtensorMap& mcr, const TileParams& p,
+                        cudaStream_t s) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(quantize_tile_kernel<SR_T, DUAL, SR_R, SWZ>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kTileSmem);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  dim3 grid((unsigned)ceil_div(p.cols, kTileCols), (unsigned)ceil_div(p.rows, kTileRows));
+  quantize_tile_kernel<SR_T, DUAL, SR_R, SWZ><<<grid, kThreads, kTileSmem, s>>>(mx, mct, mcr, p);
+  return cudaGetLastError();
+}
+
+template <bool DUAL, bool SWZ>
+cudaError_t dispatch_tile(bool sr_t, bool sr_r, const CUtensorMap& mx, const CUtensorMap& mct, const CUtensorMap& mcr,
+                          const TileParams& p, cudaStream_t s) {
+  if constexpr (DUAL) {
+    if (sr_t) return sr_r ? launch_tile<true, true, true, SWZ>(mx, mct, mcr, p, s) : launch_tile<true, true, false, SWZ>(mx, mct, mcr, p, s);
+    return sr_r ? launch_tile<false, true, true, SWZ>(mx, mct, mcr, p, s) : launch_tile<false, true, false, SWZ>(mx, mct, mcr, p, s);
+  } else {
+    return sr_t ? launch_tile<true, false, false, SWZ>(mx, mct, mcr, p, s) : launch_tile<false, false, false, SWZ>(mx, mct, mcr, p, s);
+  }
+}
+
+}  // namespace
+
+// True when the tile kernel can take the tensor: bf16, rows a multiple of 32 (16-byte pitch of the
+// transposed codes) and, for the row output, columns a multiple of 32 as well.
+bool tile_quantizer_eligible(int dtype, int64_t rows, int64_t cols, bool dual) {
+  if (dtype != NVFP4_BF16 || rows % 32 != 0) return false;
+  if (dual && cols % 32 != 0) return false;
+  if (ceil_div(rows, kTileRows) > 65535) return false;      // grid.y limit
+  return true;
+}
+
+// Launches the tile kernel.  r_* arguments are ignored unless `dual`.  Arguments are validated by the callers.
+int tile_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, const float* g, bool dual,
+                  const nvfp4_rounding* rt, uint8_t* codes_t, uint8_t* scales_t,
+                  const nvfp4_rounding* rr, uint8_t* codes_r, uint8_t* scales_r, int sf_layout, cudaStream_t s) {
+  CUtensorMap mx, mct, mcr;
+  if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, x, (uint64_t)cols, (uint64_t)rows, (uint64_t)ld * 2, kTileCols,
+                   kTileRows, CU_TENSOR_MAP_SWIZZLE_128B))
+    return NVFP4_ERR_CUDA;
+  if (!make_map_2d(&mct, CU_TENSOR_MAP_DATA_TYPE_UINT8, codes_t, (uint64_t)rows / 2, (uint64_t)cols, (uint64_t)rows / 2,
+                   kTileRows / 2, kTileCols, CU_TENSOR_MAP_SWIZZLE_128B))
+    return NVFP4_ERR_CUDA;
+  mcr = mct;
+  if (dual && !make_map_2d(&mcr, CU_TENSOR_MAP_DATA_TYPE_UINT8, codes_r, (uint64_t)cols / 2, (uint64_t)rows,
+                           (uint64_t)cols / 2, kTileCols / 2, kTileRows, CU_TENSOR_MAP_SWIZZLE_NONE))
+    return NVFP4_ERR_CUDA;
+  TileParams p;
+  p.gptr = g; p.rows = rows; p.cols = cols;
+  p.t_seed_lo = (uint32_t)rt->seed; p.t_seed_hi = (uint32_t)(rt->seed >> 32);
+  p.t_off_lo = (uint32_t)rt->offset; p.t_off_hi = (uint32_t)(rt->offset >> 32);
+  p.t_scales = scales_t; p.t_nkb = rows / 16; p.t_k_tiles = ceil_div(p.t_nkb, 4);
+  const nvfp4_rounding* r2 = dual ? rr : rt;
+  p.r_seed_lo = (uint32_t)r2->seed; p.r_seed_hi = (uint32_t)(r2->seed >> 32);
+  p.r_off_lo = (uint32_t)r2->offset; p.r_off_hi = (uint32_t)(r2->offset >> 32);
+  p.r_scales = scales_r; p.r_nkb = cols / 16; p.r_k_tiles = ceil_div(p.r_nkb, 4);
+  const bool swz = sf_layout == NVFP4_SF_SWIZZLED_128x4;
+  const bool sr_t = rt->mode == NVFP4_SR, sr_r = dual && rr->mode == NVFP4_SR;
+  cudaError_t e;
+  if (dual) e = swz ? dispatch_tile<true, true>(sr_t, sr_r, mx, mct, mcr, p, s) : dispatch_tile<true, false>(sr_t, sr_r, mx, mct, mcr, p, s);
+  else e = swz ? dispatch_tile<false, true>(sr_t, sr_r, mx, mct, mcr, p, s) : dispatch_tile<false, false>(sr_t, sr_r, mx, mct, mcr, p, s);
+  return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+// Reads and clears this file's device error word (set when a tile wait ran out).
+int tile_error_word(unsigned int* out) {
+  unsigned int w = 0, zero = 0;
+  if (cudaMemcpyFromSymbol(&w, g_tile_error_word, sizeof(w)) != cudaSuccess) return NVFP4_ERR_CUDA;
+  if (w != 0 && cudaMemcpyToSymbol(g_tile_error_word, &zero, sizeof(zero)) != cudaSuccess) return NVFP4_ERR_CUDA;
+  *out = w;
+  return NVFP4_OK;
+}
+
+}  // namespace nvfp4

@@ -30,7 +30,7 @@ def _time(fn, iters, warmup):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["gemm", "quantize", "amax"])
+    ap.add_argument("kernel", choices=["gemm", "quantize", "dual", "amax"])
     ap.add_argument("--m", type=int, default=8192)
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--k", type=int, default=4096)
@@ -74,6 +74,23 @@ def main():
         nbytes = a.rows * a.cols * (x.element_size() + 0.5625)
         res = {"kernel": "quantize", "rows": a.rows, "cols": a.cols, "transposed": a.transposed, "sr": a.sr,
                "dtype": str(dt), "ms": ms, "GB/s": nbytes / ms / 1e6}
+    elif a.kernel == "dual":
+        x = synth.heavy_tailed((a.rows, a.cols), 1002, device=dev)
+        g = nb.nvfp4_tensor_amax_scale(x)
+        r = nb.Rounding(nb.SR, 1, 0) if a.sr else nb.Rounding()
+        r2 = nb.Rounding(nb.SR, 1, 1) if a.sr else nb.Rounding()
+        L = nb.lib()
+        cr, sr_, ct, st_ = nb.nvfp4_quantize_dual(x, g, r, r2, nb.SF_SWIZZLED)
+
+        def run():
+            import ctypes as C
+            s = L.nvfp4_quantize_dual(x.data_ptr(), 0, a.rows, a.cols, x.stride(0), g.data_ptr(), C.byref(r), cr.data_ptr(),
+                                      sr_.data_ptr(), C.byref(r2), ct.data_ptr(), st_.data_ptr(), nb.SF_SWIZZLED,
+                                      torch.cuda.current_stream().cuda_stream)
+            assert s == 0
+        ms = _time(run, a.iters, a.warmup)
+        res = {"kernel": "dual", "rows": a.rows, "cols": a.cols, "sr": a.sr, "ms": ms,
+               "GB/s": a.rows * a.cols * 3.125 / ms / 1e6}
     else:
         x = synth.normal((a.rows, a.cols), 1.0, 3, device=dev)
         out = torch.empty(1, dtype=torch.float32, device=dev)

@@ -10,7 +10,8 @@ from tests.util import assert_quantize_parity
 pytestmark = pytest.mark.gpu
 
 ROW_SHAPES = [(1, 16), (3, 48), (130, 80), (128, 512), (257, 1040), (256, 512), (129, 4112)]
-T_SHAPES = [(16, 8), (48, 24), (272, 72), (512, 200), (256, 64), (1040, 264), (4112, 136)]
+# rows % 32 == 0 takes the tiled-copy kernel (ragged tiles in both directions), the others the fallback kernel
+T_SHAPES = [(16, 8), (48, 24), (272, 72), (512, 200), (256, 64), (1040, 264), (4112, 136), (288, 72), (32, 8), (1056, 328)]
 
 
 def _x(shape, seed, dtype=torch.bfloat16, std=1.0):
@@ -97,3 +98,41 @@ def test_strided_input():
 def test_heavy_tailed_sweep(n_elem, transposed, mode):
     x = synth.heavy_tailed(synth.square_shape(n_elem), seed=1001, device="cpu").cuda()
     assert_quantize_parity(x, transposed, True, nb.Rounding(mode, 1, 0), nb.SF_SWIZZLED)
+
+
+# ---------------------------------------------------------------- both orientations from one read
+DUAL_SHAPES = [(256, 64), (512, 192), (288, 96), (32, 32), (1056, 352), (48, 80), (272, 48)]   # the last two: fallback path
+
+
+@pytest.mark.parametrize("sf_layout", [nb.SF_LINEAR, nb.SF_SWIZZLED])
+@pytest.mark.parametrize("modes", [(nb.RTN, nb.SR), (nb.SR, nb.SR), (nb.RTN, nb.RTN), (nb.SR, nb.RTN)])
+@pytest.mark.parametrize("shape", DUAL_SHAPES)
+def test_dual_matches_the_oracle_in_both_orientations(shape, modes, sf_layout):
+    from oracle import binding as ob
+    from tests.util import oracle_quantize
+    x = _x(shape, 11)
+    g_t = nb.nvfp4_tensor_amax_scale(x)
+    g = float(g_t.item())
+    rr, rt = nb.Rounding(modes[0], 21, 4), nb.Rounding(modes[1], 21, 5)
+    cr, sr, ct, st = nb.nvfp4_quantize_dual(x, g_t, rr, rt, sf_layout)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
+    for got_c, got_s, transposed, r in ((cr, sr, False, rr), (ct, st, True, rt)):
+        oc, osf = oracle_quantize(x, transposed, g, r)
+        if sf_layout == nb.SF_SWIZZLED:
+            osf = ob.sf_swizzle(osf)
+        assert np.array_equal(got_c.cpu().numpy(), oc)
+        assert np.array_equal(got_s.cpu().numpy().reshape(-1), osf.reshape(-1))
+
+
+def test_dual_heavy_tailed_2p24():
+    from oracle import binding as ob
+    from tests.util import oracle_quantize
+    x = synth.heavy_tailed(synth.square_shape(2 ** 24), seed=1001, device="cpu").cuda()
+    g_t = nb.nvfp4_tensor_amax_scale(x)
+    rr, rt = nb.Rounding(nb.SR, 1, 0), nb.Rounding(nb.SR, 1, 1)
+    cr, sr, ct, st = nb.nvfp4_quantize_dual(x, g_t, rr, rt, nb.SF_SWIZZLED)
+    for got_c, got_s, transposed, r in ((cr, sr, False, rr), (ct, st, True, rt)):
+        oc, osf = oracle_quantize(x, transposed, float(g_t.item()), r)
+        assert np.array_equal(got_c.cpu().numpy(), oc)
+        assert np.array_equal(got_s.cpu().numpy().reshape(-1), ob.sf_swizzle(osf).reshape(-1))
