@@ -202,19 +202,27 @@ def main():
                            Y=torch.empty((M, N), dtype=torch.float32, device=dev),
                            dX=torch.empty((M, K), dtype=torch.float32, device=dev),
                            dW=torch.empty((N, K), dtype=torch.float32, device=dev)))
-    ws_bytes = max(nb.nvfp4_linear_workspace_bytes(M, l["N"], l["K"], w) for l in layers for w in (0, 1, 2))
+    ws_bytes = max(nb.nvfp4_linear_fused_workspace_bytes(M, l["N"], l["K"], w) for l in layers
+                   for w in (nb.FUSED_FWD_SAVE, nb.FUSED_BWD_SAVED))
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+    saved = torch.empty(max(nb.nvfp4_linear_saved_bytes(M, l["N"], l["K"]) for l in layers), dtype=torch.uint8, device=dev)
     rt = nb.Rounding(nb.RTN)
     sr = [nb.Rounding(nb.SR, 0, o) for o in range(3)]      # distinct offsets per SR site
     in_bytes = sum(t.numel() * t.element_size() for l in layers for t in (l["X"], l["W"], l["dY"]))
 
+    def layer_fwd_bwd(l):
+        # forward (Eq. 1/4) keeping Q(X^T), Q(W^T); backward + update (Eq. 2/5, 3/6) from one read of dY.
+        # Each tensor's amax is taken once, each tensor is read once per pass.
+        nb.nvfp4_linear_fwd_save(l["X"], l["W"], nb.G_AMAX, rx=rt, rw=rt, rxt=sr[2], rwt=rt, out=l["Y"], saved=saved,
+                                 workspace=ws)
+        nb.nvfp4_linear_bwd_saved(l["dY"], saved, l["K"], nb.G_AMAX, rdy=sr[0], rdyt=sr[1], dX=l["dX"], dW=l["dW"],
+                                  workspace=ws)
+
     def step():
         for l in layers:
-            nb.nvfp4_linear_fwd(l["X"], l["W"], nb.G_AMAX, rx=rt, rw=rt, out=l["Y"], workspace=ws)
-            nb.nvfp4_linear_bwd_dx(l["dY"], l["W"], nb.G_AMAX, rdy=sr[0], rw=rt, out=l["dX"], workspace=ws)
-            nb.nvfp4_linear_bwd_dw(l["dY"], l["X"], nb.G_AMAX, rdy=sr[1], rx=sr[2], out=l["dW"], workspace=ws)
+            layer_fwd_bwd(l)
 
-    launches_per_step = len(layers) * 3 * 7       # 2 x (amax + finalize) + 2 quantize + 1 GEMM per product
+    launches_per_step = len(layers) * (3 * 2 + 3 + 3)     # 3 x (amax + finalize), 3 dual quantizers, 3 GEMMs per layer
     flops_per_step = block_flops(cfg)
 
     def barrier():
@@ -335,9 +343,7 @@ def main():
             for l, h in zip(layers, host_in):
                 for k in ("X", "W", "dY"):
                     l[k].copy_(h[k], non_blocking=True)
-                nb.nvfp4_linear_fwd(l["X"], l["W"], nb.G_AMAX, rx=rt, rw=rt, out=l["Y"], workspace=ws)
-                nb.nvfp4_linear_bwd_dx(l["dY"], l["W"], nb.G_AMAX, rdy=sr[0], rw=rt, out=l["dX"], workspace=ws)
-                nb.nvfp4_linear_bwd_dw(l["dY"], l["X"], nb.G_AMAX, rdy=sr[1], rx=sr[2], out=l["dW"], workspace=ws)
+                layer_fwd_bwd(l)
                 for k in ("Y", "dX", "dW"):
                     host_out[k][:l[k].numel()].copy_(l[k].view(-1), non_blocking=True)
 
@@ -382,7 +388,8 @@ def main():
             "config": {"workload": "llama7b_block_linears_fwd_bwd" if args.workload == "llama7b" else "llama350m_block_linears_fwd_bwd",
                        "tokens": M, "hidden": cfg["hidden"], "linears": [[n, k, o] for n, k, o in cfg["linears"]],
                        "products_per_step": 15, "rounding": "RtN forward, Philox SR backward/update",
-                       "per_tensor_scale": "amax/(6*448), computed inside every call",
+                       "per_tensor_scale": "amax/(6*448), computed once per tensor inside the calls",
+                       "fusion": "nvfp4_linear_fwd_save + nvfp4_linear_bwd_saved: X, W, dY each read once per pass, both orientations quantized from that read",
                        "l2": f"inputs exceed L2: {in_bytes / 2 ** 20:.0f} MiB of operands per step, fp32 outputs on top",
                        "parallelism": "replicas only (one GPU per rank, no data-path collective)"},
             "pct_of_fp4_peak": {"of_nominal_9pf": value / world / 9000.0 * 100,

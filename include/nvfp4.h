@@ -178,6 +178,45 @@ NVFP4_API int nvfp4_linear_bwd_dw(const void* dY, const void* X, int dtype, int6
                         void* dW, int dw_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * The layer of Eq. 1-6 with every tensor read once per pass (fused producers).
+ *
+ * Eq. 4-6 use X, W and dY in both orientations.  nvfp4_linear_fwd_save computes Y as
+ * nvfp4_linear_fwd does and, from the same reads of X and W, also writes Q(X^T) (rounding rxt; the
+ * paper: SR, Eq. 6) and Q(W^T) (rounding rwt; the paper: RtN, Eq. 5) with their per-tensor scales
+ * into `saved`.  nvfp4_linear_bwd_saved then needs only dY: it quantizes it both ways from one read
+ * (rdy for Q(dY) of Eq. 5, rdyt for Q(dY^T) of Eq. 6) and runs both GEMMs, dX[M,K] and dW[N,K].
+ * nvfp4_linear_bwd is the same backward + update pass without saved state (it quantizes W^T and X^T
+ * itself).  With equal rounding arguments all results equal those of nvfp4_linear_fwd /
+ * nvfp4_linear_bwd_dx / nvfp4_linear_bwd_dw bit for bit.
+ *
+ * M, N, K must be multiples of 32.  `saved`: nvfp4_linear_saved_bytes(M,N,K) bytes, 256-byte
+ * aligned, owned by the caller, written by fwd_save and only read by bwd_saved (which must be given
+ * the same gscale_mode).  workspace: nvfp4_linear_fused_workspace_bytes(M,N,K,which) bytes, 256-byte
+ * aligned, contents undefined afterwards.  gscale_mode as in nvfp4_linear_fwd.
+ */
+typedef enum { NVFP4_FUSED_FWD_SAVE = 0, NVFP4_FUSED_BWD_SAVED = 1, NVFP4_FUSED_BWD = 2 } nvfp4_fused_kind;
+NVFP4_API size_t nvfp4_linear_saved_bytes(int64_t M, int64_t N, int64_t K);
+NVFP4_API size_t nvfp4_linear_fused_workspace_bytes(int64_t M, int64_t N, int64_t K, int which);
+NVFP4_API int nvfp4_linear_fwd_save(const void* X, const void* W, int dtype, int64_t M, int64_t N, int64_t K,
+                          int gscale_mode, const float* gx, const float* gw,
+                          const nvfp4_rounding* rx, const nvfp4_rounding* rw,
+                          const nvfp4_rounding* rxt, const nvfp4_rounding* rwt,
+                          void* Y, int y_dtype, void* saved, size_t saved_bytes,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+NVFP4_API int nvfp4_linear_bwd_saved(const void* dY, int dtype, int64_t M, int64_t N, int64_t K,
+                           int gscale_mode, const float* gdy,
+                           const nvfp4_rounding* rdy, const nvfp4_rounding* rdyt,
+                           const void* saved, size_t saved_bytes,
+                           void* dX, int dx_dtype, void* dW, int dw_dtype,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+NVFP4_API int nvfp4_linear_bwd(const void* dY, const void* W, const void* X, int dtype, int64_t M, int64_t N, int64_t K,
+                     int gscale_mode, const float* gdy, const float* gw, const float* gx,
+                     const nvfp4_rounding* rdy, const nvfp4_rounding* rdyt,
+                     const nvfp4_rounding* rwt, const nvfp4_rounding* rxt,
+                     void* dX, int dx_dtype, void* dW, int dw_dtype,
+                     void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * nvfp4_linear_fwd without a caller-supplied workspace and without any device-memory
  * allocation (the paper has no counterpart; this is a library convenience).
  *

@@ -67,6 +67,16 @@ def lib():
     for name in ("nvfp4_linear_fwd", "nvfp4_linear_bwd_dx", "nvfp4_linear_bwd_dw"):
         getattr(L, name).restype = ci
         getattr(L, name).argtypes = lin
+    L.nvfp4_linear_saved_bytes.restype = sz
+    L.nvfp4_linear_saved_bytes.argtypes = [i64, i64, i64]
+    L.nvfp4_linear_fused_workspace_bytes.restype = sz
+    L.nvfp4_linear_fused_workspace_bytes.argtypes = [i64, i64, i64, ci]
+    L.nvfp4_linear_fwd_save.restype = ci
+    L.nvfp4_linear_fwd_save.argtypes = [vp, vp, ci, i64, i64, i64, ci, vp, vp, rp, rp, rp, rp, vp, ci, vp, sz, vp, sz, vp]
+    L.nvfp4_linear_bwd_saved.restype = ci
+    L.nvfp4_linear_bwd_saved.argtypes = [vp, ci, i64, i64, i64, ci, vp, rp, rp, vp, sz, vp, ci, vp, ci, vp, sz, vp]
+    L.nvfp4_linear_bwd.restype = ci
+    L.nvfp4_linear_bwd.argtypes = [vp, vp, vp, ci, i64, i64, i64, ci, vp, vp, vp, rp, rp, rp, rp, vp, ci, vp, ci, vp, sz, vp]
     L.nvfp4_linear_fwd_static.restype = ci
     L.nvfp4_linear_fwd_static.argtypes = [vp, vp, ci, i64, i64, i64, ci, vp, vp, rp, rp, vp, ci, vp]
     L.nvfp4_device_error_word.restype = ci
@@ -216,6 +226,75 @@ def nvfp4_linear_bwd_dw(dY, X, gscale_mode=G_AMAX, gdy=None, gx=None, rdy=None, 
     (M, N), K = dY.shape, X.shape[1]
     return _linear("nvfp4_linear_bwd_dw", LINEAR_BWD_DW, dY, X, M, N, K, (N, K), gscale_mode, gdy, gx,
                    rdy or Rounding(SR, 0, 1), rx or Rounding(SR, 0, 2), out, out_dtype, workspace, stream)
+
+
+FUSED_FWD_SAVE, FUSED_BWD_SAVED, FUSED_BWD = 0, 1, 2
+
+
+def nvfp4_linear_saved_bytes(M, N, K) -> int:
+    return int(lib().nvfp4_linear_saved_bytes(M, N, K))
+
+
+def nvfp4_linear_fused_workspace_bytes(M, N, K, which) -> int:
+    return int(lib().nvfp4_linear_fused_workspace_bytes(M, N, K, which))
+
+
+def _scratch(nbytes, device, given):
+    if given is not None:
+        return given
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+def nvfp4_linear_fwd_save(X, W, gscale_mode=G_AMAX, gx=None, gw=None, rx=None, rw=None, rxt=None, rwt=None, out=None,
+                          out_dtype=torch.float32, saved=None, workspace=None, stream=None):
+    """Y = Q(X) . Q(W)^T and, from the same reads, Q(X^T) and Q(W^T) into `saved` for the backward
+    and update passes.  Returns (Y, saved).  Default rounding: the paper's (RtN, RtN, SR for X^T, RtN for W^T)."""
+    (M, K), N = X.shape, W.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=X.device)
+    saved = _scratch(nvfp4_linear_saved_bytes(M, N, K), X.device, saved)
+    ws = _scratch(nvfp4_linear_fused_workspace_bytes(M, N, K, FUSED_FWD_SAVE), X.device, workspace)
+    st = lib().nvfp4_linear_fwd_save(_ptr(X), _ptr(W), _dtype_code(X), M, N, K, gscale_mode, _ptr(gx), _ptr(gw),
+                                     C.byref(rx or Rounding(RTN)), C.byref(rw or Rounding(RTN)),
+                                     C.byref(rxt or Rounding(SR, 0, 2)), C.byref(rwt or Rounding(RTN)),
+                                     _ptr(out), _dtype_code(out), _ptr(saved), saved.numel(), _ptr(ws), ws.numel(),
+                                     _stream(stream))
+    _check(st, "nvfp4_linear_fwd_save")
+    return out, saved
+
+
+def nvfp4_linear_bwd_saved(dY, saved, K, gscale_mode=G_AMAX, gdy=None, rdy=None, rdyt=None, dX=None, dW=None,
+                           dx_dtype=torch.float32, dw_dtype=torch.float32, workspace=None, stream=None):
+    """dX and dW from one read of dY and the operands nvfp4_linear_fwd_save kept.  Returns (dX, dW)."""
+    M, N = dY.shape
+    if dX is None:
+        dX = torch.empty((M, K), dtype=dx_dtype, device=dY.device)
+    if dW is None:
+        dW = torch.empty((N, K), dtype=dw_dtype, device=dY.device)
+    ws = _scratch(nvfp4_linear_fused_workspace_bytes(M, N, K, FUSED_BWD_SAVED), dY.device, workspace)
+    st = lib().nvfp4_linear_bwd_saved(_ptr(dY), _dtype_code(dY), M, N, K, gscale_mode, _ptr(gdy),
+                                      C.byref(rdy or Rounding(SR, 0, 0)), C.byref(rdyt or Rounding(SR, 0, 1)),
+                                      _ptr(saved), saved.numel(), _ptr(dX), _dtype_code(dX), _ptr(dW), _dtype_code(dW),
+                                      _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "nvfp4_linear_bwd_saved")
+    return dX, dW
+
+
+def nvfp4_linear_bwd(dY, W, X, gscale_mode=G_AMAX, gdy=None, gw=None, gx=None, rdy=None, rdyt=None, rwt=None, rxt=None,
+                     dX=None, dW=None, dx_dtype=torch.float32, dw_dtype=torch.float32, workspace=None, stream=None):
+    """dX and dW (Eq. 2/5 and Eq. 3/6) with dY read once.  Returns (dX, dW)."""
+    (M, N), K = dY.shape, W.shape[1]
+    if dX is None:
+        dX = torch.empty((M, K), dtype=dx_dtype, device=dY.device)
+    if dW is None:
+        dW = torch.empty((N, K), dtype=dw_dtype, device=dY.device)
+    ws = _scratch(nvfp4_linear_fused_workspace_bytes(M, N, K, FUSED_BWD), dY.device, workspace)
+    st = lib().nvfp4_linear_bwd(_ptr(dY), _ptr(W), _ptr(X), _dtype_code(dY), M, N, K, gscale_mode, _ptr(gdy), _ptr(gw),
+                                _ptr(gx), C.byref(rdy or Rounding(SR, 0, 0)), C.byref(rdyt or Rounding(SR, 0, 1)),
+                                C.byref(rwt or Rounding(RTN)), C.byref(rxt or Rounding(SR, 0, 2)),
+                                _ptr(dX), _dtype_code(dX), _ptr(dW), _dtype_code(dW), _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "nvfp4_linear_bwd")
+    return dX, dW
 
 
 STATIC_WORKSPACE_BYTES = 8 << 20

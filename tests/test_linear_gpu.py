@@ -114,3 +114,42 @@ def test_350m_block_linears_sampled(name, K, N):
     s = sample(N, K)
     _assert_close(_host(dW)[s[0], s[1]], *oracle_linear("dw", dY, X, sr1, sr2, True, s))
     assert nb.nvfp4_device_error_word() == 0
+
+
+# ---------------------------------------------------------------- fused layer: every tensor read once per pass
+@pytest.mark.parametrize("use_g", [True, False])
+@pytest.mark.parametrize("shape", [(256, 512, 512), (160, 288, 224), (512, 64, 96)])
+def test_fused_layer_equals_the_separate_products(shape, use_g):
+    M, K, N = shape
+    X, W, dY = synth.linear_inputs(M, K, N, seed=31, grad_std=1e-3)
+    X, W, dY = X.cuda(), W.cuda(), dY.cuda()
+    mode = nb.G_AMAX if use_g else nb.G_NONE
+    rt, sr0, sr1, sr2 = nb.Rounding(nb.RTN), nb.Rounding(nb.SR, 5, 0), nb.Rounding(nb.SR, 5, 1), nb.Rounding(nb.SR, 5, 2)
+    Y = nb.nvfp4_linear_fwd(X, W, gscale_mode=mode, rx=rt, rw=rt)
+    dX = nb.nvfp4_linear_bwd_dx(dY, W, gscale_mode=mode, rdy=sr0, rw=rt)
+    dW = nb.nvfp4_linear_bwd_dw(dY, X, gscale_mode=mode, rdy=sr1, rx=sr2)
+    Yf, saved = nb.nvfp4_linear_fwd_save(X, W, gscale_mode=mode, rx=rt, rw=rt, rxt=sr2, rwt=rt)
+    dXf, dWf = nb.nvfp4_linear_bwd_saved(dY, saved, K, gscale_mode=mode, rdy=sr0, rdyt=sr1)
+    dXb, dWb = nb.nvfp4_linear_bwd(dY, W, X, gscale_mode=mode, rdy=sr0, rdyt=sr1, rwt=rt, rxt=sr2)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
+    assert torch.equal(Y, Yf) and torch.equal(dX, dXf) and torch.equal(dW, dWf)
+    assert torch.equal(dX, dXb) and torch.equal(dW, dWb)
+    _assert_close(_host(Yf), *oracle_linear("fwd", X, W, rt, rt, use_g))
+    _assert_close(_host(dXf), *oracle_linear("dx", dY, W, sr0, rt, use_g))
+    _assert_close(_host(dWf), *oracle_linear("dw", dY, X, sr1, sr2, use_g))
+
+
+def test_fused_layer_with_given_scales_and_bf16_outputs():
+    M, K, N = 256, 256, 384
+    X, W, dY = synth.linear_inputs(M, K, N, seed=32, grad_std=1e-3)
+    X, W, dY = X.cuda(), W.cuda(), dY.cuda()
+    gx, gw, gdy = (nb.nvfp4_tensor_amax_scale(t) for t in (X, W, dY))
+    Y, saved = nb.nvfp4_linear_fwd_save(X, W, gscale_mode=nb.G_GIVEN, gx=gx, gw=gw, out_dtype=torch.bfloat16)
+    dX, dW = nb.nvfp4_linear_bwd_saved(dY, saved, K, gscale_mode=nb.G_GIVEN, gdy=gdy, dx_dtype=torch.bfloat16)
+    rt = nb.Rounding(nb.RTN)
+    ref, T = oracle_linear("fwd", X, W, rt, rt, True)
+    assert np.all(np.abs(_host(Y) - ref) <= TOL * T + np.abs(ref) * 2.0 ** -8)
+    ref, T = oracle_linear("dx", dY, W, nb.Rounding(nb.SR, 0, 0), rt, True)
+    assert np.all(np.abs(_host(dX) - ref) <= TOL * T + np.abs(ref) * 2.0 ** -8)
+    _assert_close(_host(dW), *oracle_linear("dw", dY, X, nb.Rounding(nb.SR, 0, 1), nb.Rounding(nb.SR, 0, 2), True))
