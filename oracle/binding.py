@@ -43,6 +43,8 @@ def lib():
         q = [_f32p, C.c_int64, C.c_int64, C.c_float, C.c_int, C.c_uint64, C.c_uint64, _u8p, _u8p, C.c_int]
         L.nvfp4o_quantize.restype = None
         L.nvfp4o_quantize.argtypes = q
+        L.nvfp4o_quantize_rows.restype = None
+        L.nvfp4o_quantize_rows.argtypes = q[:7] + [C.c_int64] + q[7:]
         L.nvfp4o_quantize_transposed.restype = None
         L.nvfp4o_quantize_transposed.argtypes = q
         L.nvfp4o_dequantize.restype = None
@@ -127,6 +129,19 @@ def quantize(x, g=1.0, mode=RTN, seed=0, offset=0, transposed=False, nthreads=No
     nt = host_threads() if nthreads is None else nthreads
     fn = lib().nvfp4o_quantize_transposed if transposed else lib().nvfp4o_quantize
     fn(x, rows, cols, float(np.float32(g)), mode, seed, offset, codes, scales, nt)
+    return codes, scales
+
+
+def quantize_rows(x, first_row, g=1.0, mode=RTN, seed=0, offset=0, nthreads=None):
+    """Row quantization of a slice x = full[first_row : first_row + x.shape[0]] of a taller tensor
+    (for a transposed quantization pass the transposed slice of columns and the first column)."""
+    x = _f32(x)
+    rows, cols = x.shape
+    assert cols % 16 == 0
+    codes = np.zeros((rows, cols // 2), dtype=np.uint8)
+    scales = np.zeros((rows, cols // 16), dtype=np.uint8)
+    nt = host_threads() if nthreads is None else nthreads
+    lib().nvfp4o_quantize_rows(x, rows, cols, float(np.float32(g)), mode, seed, offset, first_row, codes, scales, nt)
     return codes, scales
 
 

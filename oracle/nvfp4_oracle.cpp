@@ -152,6 +152,12 @@ uint8_t nvfp4o_round_sr(float y, uint16_t r16) {
 void nvfp4o_quantize(const float* x, int64_t Rq, int64_t Kq, float g, int mode,
                      uint64_t seed, uint64_t offset,
                      uint8_t* codes, uint8_t* scales, int nthreads) {
+  nvfp4o_quantize_rows(x, Rq, Kq, g, mode, seed, offset, 0, codes, scales, nthreads);
+}
+
+void nvfp4o_quantize_rows(const float* x, int64_t Rq, int64_t Kq, float g, int mode,
+                          uint64_t seed, uint64_t offset, int64_t first_row,
+                          uint8_t* codes, uint8_t* scales, int nthreads) {
   const int64_t nkb = Kq / 16;
   const float c = (1.0f / 6.0f) / g;                           // once per call: two fp32 divisions
   parallel_rows(Rq, nthreads, [=](int64_t r0, int64_t r1) {
@@ -166,7 +172,7 @@ void nvfp4o_quantize(const float* x, int64_t Rq, int64_t Kq, float g, int mode,
         float d = s_d * g;
         float inv = (s_q == 0) ? 0.0f : 1.0f / d;              // one division per block
         uint16_t rnd[16];
-        if (mode == 1) nvfp4o_block_random_u16(seed, offset, (uint64_t)(r * nkb + kb), rnd);
+        if (mode == 1) nvfp4o_block_random_u16(seed, offset, (uint64_t)((first_row + r) * nkb + kb), rnd);
         uint8_t nib[16];
         for (int j = 0; j < 16; ++j) {
           float y = std::fabs(xb[j]) * inv;

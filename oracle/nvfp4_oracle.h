@@ -64,6 +64,13 @@ void nvfp4o_quantize(const float* x, int64_t Rq, int64_t Kq, float g, int mode,
                      uint64_t seed, uint64_t offset,
                      uint8_t* codes, uint8_t* scales, int nthreads);
 
+/* The same for rows first_row .. first_row+Rq-1 of a taller tensor: x points at the slice, and
+ * the block of slice row r, block kb draws its random integers as block (first_row + r)*(Kq/16) + kb.
+ * Lets a test check a slice of a tensor too large to quantize whole on the host. */
+void nvfp4o_quantize_rows(const float* x, int64_t Rq, int64_t Kq, float g, int mode,
+                          uint64_t seed, uint64_t offset, int64_t first_row,
+                          uint8_t* codes, uint8_t* scales, int nthreads);
+
 /* Transposed quantization of x[rows, cols]: by definition nvfp4o_quantize
  * applied to the materialised transpose (Rq = cols, Kq = rows). */
 void nvfp4o_quantize_transposed(const float* x, int64_t rows, int64_t cols, float g, int mode,

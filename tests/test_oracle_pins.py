@@ -375,6 +375,15 @@ def test_quantize_sr_uses_block_indexed_integers_and_is_reproducible():
                 assert nib == (m | (8 if np.signbit(v) else 0))
 
 
+def test_quantize_rows_of_a_slice_equals_the_slice_of_the_whole():
+    rng = np.random.default_rng(12)
+    x = torch.from_numpy(rng.standard_normal((40, 64)).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    for mode in (ob.RTN, ob.SR):
+        c, s_ = ob.quantize(x, g=0.5, mode=mode, seed=3, offset=9, nthreads=1)
+        c2, s2 = ob.quantize_rows(x[17:29], 17, g=0.5, mode=mode, seed=3, offset=9, nthreads=2)
+        assert np.array_equal(c[17:29], c2) and np.array_equal(s_[17:29], s2)
+
+
 def test_quantize_transposed_is_row_quantize_of_the_transpose():
     rng = np.random.default_rng(8)
     x = torch.from_numpy(rng.standard_normal((32, 24)).astype(np.float32)).to(torch.bfloat16).float().numpy()
