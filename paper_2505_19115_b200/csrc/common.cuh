@@ -93,17 +93,35 @@ __device__ __forceinline__ uint32_t e2m1x8_rs(const float (&y)[16], int o, uint3
 // ---------------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al. 2011): key = seed, counter = (block index, offset)
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t k0, uint32_t k1, uint32_t c0, uint32_t c1,
-                                               uint32_t c2, uint32_t c3) {
+// One random stream: the ten round keys of the seed (key + i * Weyl increment, precomputed on the
+// host so that a round costs two wide multiplies and two three-way XORs) and counter words 2, 3.
+struct PhiloxStream {
+  uint32_t k0[10], k1[10];
+  uint32_t off_lo, off_hi;
+};
+
+inline void philox_stream_init(PhiloxStream* s, uint64_t seed, uint64_t offset) {
+  uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+  for (int i = 0; i < 10; ++i) {
+    s->k0[i] = k0;
+    s->k1[i] = k1;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  s->off_lo = (uint32_t)offset;
+  s->off_hi = (uint32_t)(offset >> 32);
+}
+
+// Counter = (c0, c1, off_lo, off_hi); c0, c1 = the block's linear index.
+__device__ __forceinline__ uint4 philox4x32_10(const PhiloxStream& s, uint32_t c0, uint32_t c1) {
+  uint32_t c2 = s.off_lo, c3 = s.off_hi;
 #pragma unroll
   for (int i = 0; i < 10; ++i) {
     const uint64_t p0 = (uint64_t)c0 * 0xD2511F53ull, p1 = (uint64_t)c2 * 0xCD9E8D57ull;   // one wide multiply each
-    c0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
-    c2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    c0 = (uint32_t)(p1 >> 32) ^ c1 ^ s.k0[i];
+    c2 = (uint32_t)(p0 >> 32) ^ c3 ^ s.k1[i];
     c1 = (uint32_t)p1;
     c3 = (uint32_t)p0;
-    k0 += 0x9E3779B9u;
-    k1 += 0xBB67AE85u;
   }
   return make_uint4(c0, c1, c2, c3);
 }

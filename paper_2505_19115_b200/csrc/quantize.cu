@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(kThreads, 3) quantize_row_kernel(const QuantPa
       float v[16];
       const float amax = raw[u].unpack(v);
       uint32_t lo, hi, sf;
-      encode_block<SR>(v, amax, c, inv_table, p, (uint64_t)(r * p.nkb + kb), lo, hi, sf);
+      encode_block<SR>(v, amax, c, inv_table, p.rng, (uint64_t)(r * p.nkb + kb), lo, hi, sf);
       *reinterpret_cast<uint2*>(p.codes + (r * p.nkb + kb) * 8) = make_uint2(lo, hi);
       if constexpr (SWZ) {
         sf_s[(lane >> 2) * kSfChunkPitch + (rl & 31) * 16 + (rl >> 5) * 4 + (lane & 3)] = (uint8_t)sf;
@@ -173,10 +173,10 @@ __global__ void __launch_bounds__(kThreads, 3) quantize_transposed_kernel(const 
     const int64_t kb = r0 / 16 + rb;
     const int64_t ca = c0 + 2 * lane;
     uint32_t lo, hi, sf;
-    encode_block<SR>(va, amax_a, c, inv_table, p, (uint64_t)(ca * p.nkb + kb), lo, hi, sf);
+    encode_block<SR>(va, amax_a, c, inv_table, p.rng, (uint64_t)(ca * p.nkb + kb), lo, hi, sf);
     *reinterpret_cast<uint2*>(code_s + lane * TT::kCodePitch + rb * 8) = make_uint2(lo, hi);
     sf_s[rb * kTCols + lane] = (uint8_t)sf;
-    encode_block<SR>(vb, amax_b, c, inv_table, p, (uint64_t)((ca + 1) * p.nkb + kb), lo, hi, sf);
+    encode_block<SR>(vb, amax_b, c, inv_table, p.rng, (uint64_t)((ca + 1) * p.nkb + kb), lo, hi, sf);
     *reinterpret_cast<uint2*>(code_s + (32 + lane) * TT::kCodePitch + rb * 8) = make_uint2(lo, hi);
     sf_s[rb * kTCols + 32 + lane] = (uint8_t)sf;
   }
@@ -243,6 +243,49 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const T* x, int64_t rows
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
   if ((threadIdx.x & 31) == 0 && amax > 0.0f) atomicMax(out_bits, __float_as_uint(amax));  // non-negative floats order as ints
+}
+
+// Dense tensors (ld == cols, 32-byte aligned): a flat sweep with four 256-bit loads in flight per thread.
+template <typename T>
+__global__ void __launch_bounds__(kThreads) amax_flat_kernel(const uint32_t* x, int64_t n_vec32, unsigned int* out_bits) {
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+  uint32_t mb = 0u;        // bf16: packed running |max| pair
+  float mf = 0.0f;         // fp32: running max
+  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec32; i += 4 * stride) {
+    uint32_t w[4][8];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int64_t j = i + u * stride;
+      if (j < n_vec32) {
+        asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(w[u][0]), "=r"(w[u][1]), "=r"(w[u][2]), "=r"(w[u][3]), "=r"(w[u][4]), "=r"(w[u][5]),
+                       "=r"(w[u][6]), "=r"(w[u][7])
+                     : "l"(x + j * 8));
+      } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) w[u][k] = 0u;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if constexpr (sizeof(T) == 2) {
+        mb = absmax_bf16x2(absmax_bf16x2(absmax_bf16x2(absmax_bf16x2(w[u][0], w[u][1]), absmax_bf16x2(w[u][2], w[u][3])),
+                                         absmax_bf16x2(absmax_bf16x2(w[u][4], w[u][5]), absmax_bf16x2(w[u][6], w[u][7]))),
+                           mb);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) mf = fmaxf(mf, fabsf(__uint_as_float(w[u][k])));
+      }
+    }
+  }
+  float amax = mf;
+  if constexpr (sizeof(T) == 2) {
+    mb &= 0x7FFF7FFFu;
+    amax = fmaxf(__uint_as_float(mb << 16), __uint_as_float(mb & 0xFFFF0000u));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+  if ((threadIdx.x & 31) == 0 && amax > 0.0f) atomicMax(out_bits, __float_as_uint(amax));
 }
 
 __global__ void amax_finalize_kernel(float* out) {
@@ -314,8 +357,7 @@ extern "C" int nvfp4_quantize(const void* x, int dtype, int64_t rows, int64_t co
 
   QuantParams p;
   p.x = x; p.rows = rows; p.cols = cols; p.ld = ld; p.gptr = global_scale;
-  p.seed_lo = (uint32_t)rounding->seed; p.seed_hi = (uint32_t)(rounding->seed >> 32);
-  p.off_lo = (uint32_t)rounding->offset; p.off_hi = (uint32_t)(rounding->offset >> 32);
+  philox_stream_init(&p.rng, rounding->seed, rounding->offset);
   p.codes = codes; p.scales = scales;
   p.nkb = Kq / 16; p.k_tiles = ceil_div(p.nkb, 4);
   if (ceil_div(rows, 128) > 65535) return NVFP4_ERR_SHAPE;  // grid.y limit
@@ -369,7 +411,16 @@ extern "C" int nvfp4_tensor_amax_scale(const void* x, int dtype, int64_t rows, i
   if (blocks > 148 * 16) blocks = 148 * 16;
   if (blocks < 1) blocks = 1;
   unsigned int* bits = reinterpret_cast<unsigned int*>(global_scale_out);
-  if (dtype == NVFP4_BF16)
+  const int64_t total_bytes = rows * cols * (dtype == NVFP4_BF16 ? 2 : 4);
+  if (ld == cols && (reinterpret_cast<uintptr_t>(x) & 31u) == 0 && total_bytes % 32 == 0) {
+    const int64_t n32 = total_bytes / 32;
+    int64_t fb = ceil_div(n32, (int64_t)kThreads * 4);
+    if (fb > 148 * 8) fb = 148 * 8;
+    if (dtype == NVFP4_BF16)
+      amax_flat_kernel<__nv_bfloat16><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, bits);
+    else
+      amax_flat_kernel<float><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, bits);
+  } else if (dtype == NVFP4_BF16)
     amax_kernel<__nv_bfloat16><<<(unsigned)blocks, kThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(x), rows, cols, ld, bits);
   else
     amax_kernel<float><<<(unsigned)blocks, kThreads, 0, s>>>(static_cast<const float*>(x), rows, cols, ld, bits);

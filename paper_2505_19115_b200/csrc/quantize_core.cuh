@@ -14,7 +14,7 @@ struct QuantParams {
   const void* x;
   int64_t rows, cols, ld;
   const float* gptr;
-  uint32_t seed_lo, seed_hi, off_lo, off_hi;
+  PhiloxStream rng;
   uint8_t* codes;
   uint8_t* scales;
   int64_t nkb;      // blocks per quantized row (Kq / 16)
@@ -32,7 +32,7 @@ __device__ __forceinline__ void build_inv_table(float* inv_table, float g) {
 // and one scale byte.  c = (1/6)/g.  `blk` is the block's linear index (Philox counter).
 template <bool SR>
 __device__ __forceinline__ void encode_block(const float (&v)[16], float amax, float c, const float* inv_table,
-                                             const QuantParams& p, uint64_t blk,
+                                             const PhiloxStream& rng, uint64_t blk,
                                              uint32_t& lo, uint32_t& hi, uint32_t& sf) {
   const uint32_t q = e4m3_encode(__fmul_rn(amax, c));
   const float inv = inv_table[q];
@@ -44,7 +44,7 @@ __device__ __forceinline__ void encode_block(const float (&v)[16], float amax, f
     lo = e2m1x8_rn(y, 0);
     hi = e2m1x8_rn(y, 8);
   } else {
-    const uint4 r4 = philox4x32_10(p.seed_lo, p.seed_hi, (uint32_t)blk, (uint32_t)(blk >> 32), p.off_lo, p.off_hi);
+    const uint4 r4 = philox4x32_10(rng, (uint32_t)blk, (uint32_t)(blk >> 32));
     lo = e2m1x8_rs(y, 0, r4.x, r4.y);
     hi = e2m1x8_rs(y, 8, r4.z, r4.w);
   }

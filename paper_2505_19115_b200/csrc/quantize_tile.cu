@@ -31,11 +31,11 @@ struct TileParams {
   const float* gptr;
   int64_t rows, cols;
   // transposed output (always): quantized shape (cols, rows)
-  uint32_t t_seed_lo, t_seed_hi, t_off_lo, t_off_hi;
+  PhiloxStream t_rng;
   uint8_t* t_scales;
   int64_t t_nkb, t_k_tiles;
   // row output (DUAL only): quantized shape (rows, cols)
-  uint32_t r_seed_lo, r_seed_hi, r_off_lo, r_off_hi;
+  PhiloxStream r_rng;
   uint8_t* r_scales;
   int64_t r_nkb, r_k_tiles;
 };
@@ -50,7 +50,7 @@ __device__ __forceinline__ uint32_t swz128(uint32_t row, uint32_t byte) {
 }
 
 template <bool SR_T, bool DUAL, bool SR_R, bool SWZ>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, 4)
 quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_ct,
                      const __grid_constant__ CUtensorMap map_cr, const TileParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -100,8 +100,6 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
   // ---- transposed output: lane -> columns (2*lane, 2*lane+1), warp -> row blocks ----
   // Codes are staged as [column][128 bytes] with the 128-byte swizzle the tiled store expects.
-  QuantParams qt;
-  qt.seed_lo = p.t_seed_lo; qt.seed_hi = p.t_seed_hi; qt.off_lo = p.t_off_lo; qt.off_hi = p.t_off_hi;
 #pragma unroll 1
   for (int rb = warp; rb < kTileRows / 16; rb += kThreads / 32) {
     uint32_t w[16];
@@ -122,18 +120,16 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const int64_t kb = r0 / 16 + rb;
     const int64_t ca = c0 + 2 * lane;
     uint32_t lo, hi, sf;
-    encode_block<SR_T>(va, __uint_as_float(mm << 16), c, inv_table, qt, (uint64_t)(ca * p.t_nkb + kb), lo, hi, sf);
+    encode_block<SR_T>(va, __uint_as_float(mm << 16), c, inv_table, p.t_rng, (uint64_t)(ca * p.t_nkb + kb), lo, hi, sf);
     *reinterpret_cast<uint2*>(codes_t + swz128(2 * lane, rb * 8)) = make_uint2(lo, hi);
     sf_t[rb * kTileCols + 2 * lane] = (uint8_t)sf;
-    encode_block<SR_T>(vb, __uint_as_float(mm & 0xFFFF0000u), c, inv_table, qt, (uint64_t)((ca + 1) * p.t_nkb + kb), lo, hi, sf);
+    encode_block<SR_T>(vb, __uint_as_float(mm & 0xFFFF0000u), c, inv_table, p.t_rng, (uint64_t)((ca + 1) * p.t_nkb + kb), lo, hi, sf);
     *reinterpret_cast<uint2*>(codes_t + swz128(2 * lane + 1, rb * 8)) = make_uint2(lo, hi);
     sf_t[rb * kTileCols + 2 * lane + 1] = (uint8_t)sf;
   }
 
   // ---- row output: thread -> (row, block of 16 columns); four rows per thread ----
   if constexpr (DUAL) {
-    QuantParams qr;
-    qr.seed_lo = p.r_seed_lo; qr.seed_hi = p.r_seed_hi; qr.off_lo = p.r_off_lo; qr.off_hi = p.r_off_hi;
     const int kbl = threadIdx.x & 3;                          // block within the tile's 64 columns
 #pragma unroll 1
     for (int i = 0; i < kTileRows / 64; ++i) {
@@ -146,7 +142,7 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       float v[16];
       const float amax = blk.unpack(v);
       uint32_t lo, hi, sf;
-      encode_block<SR_R>(v, amax, c, inv_table, qr, (uint64_t)((r0 + rl) * p.r_nkb + c0 / 16 + kbl), lo, hi, sf);
+      encode_block<SR_R>(v, amax, c, inv_table, p.r_rng, (uint64_t)((r0 + rl) * p.r_nkb + c0 / 16 + kbl), lo, hi, sf);
       *reinterpret_cast<uint2*>(codes_r + rl * 32 + kbl * 8) = make_uint2(lo, hi);
       if constexpr (SWZ) {
         sf_r[(rl >> 7) * 512 + (rl & 31) * 16 + ((rl >> 5) & 3) * 4 + kbl] = (uint8_t)sf;
@@ -269,12 +265,10 @@ int tile_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, const f
     return NVFP4_ERR_CUDA;
   TileParams p;
   p.gptr = g; p.rows = rows; p.cols = cols;
-  p.t_seed_lo = (uint32_t)rt->seed; p.t_seed_hi = (uint32_t)(rt->seed >> 32);
-  p.t_off_lo = (uint32_t)rt->offset; p.t_off_hi = (uint32_t)(rt->offset >> 32);
+  philox_stream_init(&p.t_rng, rt->seed, rt->offset);
   p.t_scales = scales_t; p.t_nkb = rows / 16; p.t_k_tiles = ceil_div(p.t_nkb, 4);
   const nvfp4_rounding* r2 = dual ? rr : rt;
-  p.r_seed_lo = (uint32_t)r2->seed; p.r_seed_hi = (uint32_t)(r2->seed >> 32);
-  p.r_off_lo = (uint32_t)r2->offset; p.r_off_hi = (uint32_t)(r2->offset >> 32);
+  philox_stream_init(&p.r_rng, r2->seed, r2->offset);
   p.r_scales = scales_r; p.r_nkb = cols / 16; p.r_k_tiles = ceil_div(p.r_nkb, 4);
   const bool swz = sf_layout == NVFP4_SF_SWIZZLED_128x4;
   const bool sr_t = rt->mode == NVFP4_SR, sr_r = dual && rr->mode == NVFP4_SR;
