@@ -774,21 +774,26 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
       tc_fence_after();
       const int row0 = tm * 256 + (int)rank * 128 + quarter * 32;
       const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
-      uint32_t r[kLoads][32];
+      // The MMA issuer cannot start the next tile before this accumulator is read out, so the read-out is
+      // what must finish early, not the stores: the first kHeld chunks are converted and parked in
+      // registers, the others stream through the staging buffers, the accumulator is handed back
+      // as soon as the last of them is read, and the parked chunks are stored after that.
+      constexpr int kChunks = BN / kChunkCols;
+      constexpr int kHeld = (kChunks > 3) ? 3 : kChunks - 1;
+
+      // one chunk: accumulator columns [c0, c0 + kChunkCols) -> 32 output words (scaled, converted)
+      auto read_chunk = [&](int c0, uint32_t (&w)[32]) {
+        uint32_t r[kLoads][32];
 #pragma unroll
-      for (int l = 0; l < kLoads; ++l) tmem_ld32(t_row + 32 * l, r[l]);
-#pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += kChunkCols, ++chunk_no) {
-        const uint32_t buf = my_buf + (chunk_no & 1u) * 4096u;
+        for (int l = 0; l < kLoads; ++l) tmem_ld32(t_row + c0 + 32 * l, r[l]);
         tmem_ld_wait();
 #pragma unroll
         for (int l = 0; l < kLoads; ++l) tmem_ld_pin(r[l]);
-        uint32_t w[32];
         if constexpr (BF16_OUT) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
             const __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[0][2 * e]) * alpha, __uint_as_float(r[0][2 * e + 1]) * alpha);
-            const __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[1][2 * e]) * alpha, __uint_as_float(r[1][2 * e + 1]) * alpha);
+            const __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[kLoads - 1][2 * e]) * alpha, __uint_as_float(r[kLoads - 1][2 * e + 1]) * alpha);
             w[e] = *reinterpret_cast<const uint32_t*>(&h0);
             w[16 + e] = *reinterpret_cast<const uint32_t*>(&h1);
           }
@@ -796,19 +801,15 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
 #pragma unroll
           for (int e = 0; e < 32; ++e) w[e] = __float_as_uint(__uint_as_float(r[0][e]) * alpha);
         }
-        if (c0 + kChunkCols < BN) {                 // next chunk's accumulator read overlaps this chunk's store
-#pragma unroll
-          for (int l = 0; l < kLoads; ++l) tmem_ld32(t_row + c0 + kChunkCols + 32 * l, r[l]);
-        } else {                                    // accumulator fully read: hand it back to the leader
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(lead_tempty0 + 8u * acc);
-        }
+      };
+      // stage 32 rows x 128 bytes (row = lane, eight 16-byte pieces, piece index XOR (row & 7): the
+      // 128-byte swizzle) and send them off as one tiled store
+      auto store_chunk = [&](int c0, const uint32_t (&w)[32]) {
+        const uint32_t buf = my_buf + (chunk_no & 1u) * 4096u;
         if (chunk_no >= 2) {                        // the store issued two chunks ago has read this buffer
           if (lane == 0) tma_store_wait_read<1>();
           __syncwarp();
         }
-        // row = lane: 128 bytes as eight 16-byte pieces, piece index XOR (row & 7) (128-byte swizzle)
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
           const uint32_t dst = buf + lane * 128 + ((c ^ (lane & 7)) << 4);
@@ -821,7 +822,25 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
           tma_store_2d(&map_d, buf, tn * BN + c0, row0);
           tma_store_commit();
         }
+        ++chunk_no;
+      };
+
+      uint32_t held[kHeld][32];
+#pragma unroll
+      for (int h = 0; h < kHeld; ++h) read_chunk(h * kChunkCols, held[h]);
+#pragma unroll 1
+      for (int c = kHeld; c < kChunks; ++c) {
+        uint32_t w[32];
+        read_chunk(c * kChunkCols, w);
+        if (c == kChunks - 1) {                     // accumulator fully read: hand it back to the leader
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(lead_tempty0 + 8u * acc);
+        }
+        store_chunk(c * kChunkCols, w);
       }
+#pragma unroll
+      for (int h = 0; h < kHeld; ++h) store_chunk(h * kChunkCols, held[h]);
       if (++acc == C::kAccStages) { acc = 0; acc_ph ^= 1u; }
     }
     if (lane == 0) tma_store_wait_all();
