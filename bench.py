@@ -27,8 +27,10 @@ from paper_2505_19115_b200 import synth  # noqa: E402
 METRIC = "NVFP4 linear fwd+bwd TFLOPS (% FP4 peak); quantizer GB/s (% HBM peak)"
 FP4_OVER_BF16 = 4.0        # nominal dense ratio: 9 PFLOP/s NVFP4 vs 2.25 PFLOP/s bf16
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram bytes per GEMM launch from the committed ncu capture (profiles/); None until measured
-GEMM_TRAFFIC_BYTES = None
+# DRAM traffic of the GEMM kernel from the committed ncu capture (profiles/gemm2_nvfp4_kernel_8192x8192x4096.md):
+# 83.7 MB read + 211.5 MB written for 306.2 MB of algorithmic bytes (operand codes and scales + fp32 output).
+# GEMM traffic follows bytes, not FLOPs, so the workload's figure is this ratio times its own algorithmic bytes.
+GEMM_TRAFFIC_RATIO = (83.73 + 211.52) / 306.2
 
 
 def load_peaks():
@@ -268,6 +270,7 @@ def main():
 
     gemm_events = []
     gemm_flops = 0.0
+    gemm_bytes = 0.0
     roof_steps = min(args.steps, 3)
     for it in range(roof_steps + 1):
         for l in layers:
@@ -282,6 +285,7 @@ def main():
                 if it > 0:                       # first pass is warm-up
                     gemm_events.append((s0, s1))
                     gemm_flops += 2.0 * out.shape[0] * out.shape[1] * ac.shape[1] * 2
+                    gemm_bytes += (ac.numel() + bc.numel()) * 1.125 + out.numel() * out.element_size()
                 del ac, asf, bc, bsf
     torch.cuda.synchronize()
     gemm_ms = sum(a.elapsed_time(b) for a, b in gemm_events)
@@ -289,8 +293,11 @@ def main():
     gemm_tflops = gemm_flops / (gemm_ms * 1e-3) / 1e12
     fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
     roofline = {
-        "bound": "tensor", "kernel": "gemm_nvfp4_kernel", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
-        "frac": gemm_tflops / fp4_peak, "traffic": GEMM_TRAFFIC_BYTES,
+        "bound": "tensor", "kernel": "gemm2_nvfp4_kernel<256>", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
+        "frac": gemm_tflops / fp4_peak, "traffic": GEMM_TRAFFIC_RATIO * gemm_bytes / n_gemm,
+        "traffic_basis": "ncu capture of an 8192x8192x4096 launch (0.96 of its algorithmic bytes), scaled by the "
+                         "algorithmic bytes per launch of this workload",
+        "algorithmic_bytes_per_launch_avg": gemm_bytes / n_gemm,
         "peak_basis": f"{peak_kind} sustained bf16 {peaks['bf16_tflops_sustained']} TFLOP/s x {FP4_OVER_BF16:g} "
                       f"(nominal dense NVFP4/bf16 ratio); burst basis {peaks['bf16_tflops'] * FP4_OVER_BF16:.0f}; nominal 9000",
         "launches": n_gemm, "avg_launch_ms": gemm_ms / n_gemm, "flops_per_launch_avg": gemm_flops / n_gemm,
@@ -322,7 +329,29 @@ def main():
             torch.cuda.synchronize()
             gbs = n_el * 2.5625 * reps / (q0.elapsed_time(q1) * 1e-3) / 1e9
             quant[label] = {"GB/s": gbs, "frac_of_measured_copy": gbs / peaks["hbm_gbs"], "frac_of_8TBs": gbs / 8000.0}
-        del xq, codes, sfs
+        # both orientations from one read (the fused layer's quantizer): 2 + 2 * 0.5625 bytes per element
+        L = nb.lib()
+        import ctypes as C
+        ct = torch.empty((xq.shape[1], xq.shape[0] // 2), dtype=torch.uint8, device=dev)
+        st = torch.empty(nb.nvfp4_sf_bytes(xq.shape[1], xq.shape[0], nb.SF_SWIZZLED), dtype=torch.uint8, device=dev)
+        for label, r1, r2 in (("dual_rtn", rt, rt), ("dual_sr", nb.Rounding(nb.SR, 1, 0), nb.Rounding(nb.SR, 1, 1))):
+            def dual():
+                stt = L.nvfp4_quantize_dual(xq.data_ptr(), nb.BF16, xq.shape[0], xq.shape[1], xq.stride(0), gq.data_ptr(),
+                                            C.byref(r1), codes.data_ptr(), sfs.data_ptr(), C.byref(r2), ct.data_ptr(),
+                                            st.data_ptr(), nb.SF_SWIZZLED, torch.cuda.current_stream().cuda_stream)
+                assert stt == 0
+            for _ in range(3):
+                dual()
+            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            q0.record()
+            for _ in range(10):
+                dual()
+            q1.record()
+            torch.cuda.synchronize()
+            gbs = n_el * 3.125 * 10 / (q0.elapsed_time(q1) * 1e-3) / 1e9
+            quant[label] = {"GB/s": gbs, "bytes_per_element": 3.125, "frac_of_measured_copy": gbs / peaks["hbm_gbs"],
+                            "frac_of_8TBs": gbs / 8000.0}
+        del xq, codes, sfs, ct, st
         torch.cuda.empty_cache()
 
     # ---- end to end through the C ABI with host buffers (H2D of every input, D2H of every output) ----
@@ -339,21 +368,55 @@ def main():
         h2d = sum(t.numel() * t.element_size() for h in host_in for t in h.values())
         d2h = sum(l[k].numel() * 4 for l in layers for k in ("Y", "dX", "dW"))
 
+        # Three streams: inputs arrive on one, the layer calls run on the second, results leave on the third,
+        # so that the PCIe transfers (full duplex) overlap each other and the compute.  Events keep the order:
+        # a layer computes after its inputs landed and after its previous outputs were read back; an input
+        # buffer is overwritten only after the layer that read it has run.
+        s_in, s_cmp, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        ev_in = [torch.cuda.Event() for _ in layers]
+        ev_done = [torch.cuda.Event() for _ in layers]
+        ev_out = [torch.cuda.Event() for _ in layers]
+        first = [True]
+
         def e2e_step():
-            for l, h in zip(layers, host_in):
-                for k in ("X", "W", "dY"):
-                    l[k].copy_(h[k], non_blocking=True)
-                layer_fwd_bwd(l)
-                for k in ("Y", "dX", "dW"):
-                    host_out[k][:l[k].numel()].copy_(l[k].view(-1), non_blocking=True)
+            for i, (l, h) in enumerate(zip(layers, host_in)):
+                with torch.cuda.stream(s_in):
+                    if not first[0]:
+                        s_in.wait_event(ev_done[i])
+                    for k in ("X", "W", "dY"):
+                        l[k].copy_(h[k], non_blocking=True)
+                    ev_in[i].record(s_in)
+                with torch.cuda.stream(s_cmp):
+                    s_cmp.wait_event(ev_in[i])
+                    if not first[0]:
+                        s_cmp.wait_event(ev_out[i])
+                    layer_fwd_bwd(l)
+                    ev_done[i].record(s_cmp)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_done[i])
+                    for k in ("Y", "dX", "dW"):
+                        host_out[k][:l[k].numel()].copy_(l[k].view(-1), non_blocking=True)
+                    ev_out[i].record(s_out)
+            first[0] = False
+
+        def e2e_join():
+            cur = torch.cuda.current_stream()
+            for st_ in (s_in, s_cmp, s_out):
+                cur.wait_stream(st_)
 
         e2e_steps = max(1, min(args.steps, 3))
+        for st_ in (s_in, s_cmp, s_out):
+            st_.wait_stream(torch.cuda.current_stream())
         e2e_step()
+        e2e_join()
         barrier()
         f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         f0.record()
+        for st_ in (s_in, s_cmp, s_out):
+            st_.wait_stream(torch.cuda.current_stream())
         for _ in range(e2e_steps):
             e2e_step()
+        e2e_join()
         f1.record()
         barrier()
         ems = f0.elapsed_time(f1)
