@@ -113,7 +113,7 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------------
 # reference arm: the CPU oracle on a bounded sample
 # ------------------------------------------------------------------------------------------------
-def oracle_sample_step(cfg, rows=32, seed=2004):
+def oracle_sample_step(cfg, rows=256, seed=2004):
     """One bounded sample of the workload on the host: the first layer's forward product for the
     first `rows` tokens (quantize those rows of X, quantize all of W, dequantize-then-matmul)."""
     from oracle import binding as ob
