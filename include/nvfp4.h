@@ -115,6 +115,18 @@ NVFP4_API int nvfp4_quantize_dual(const void* x, int dtype, int64_t rows, int64_
                         const nvfp4_rounding* rounding_t /* host */, uint8_t* codes_t, uint8_t* scales_t,
                         int sf_layout, void* cuda_stream);
 
+/*
+ * Quantization-noise monitor (Section 4): for a tensor and the quantization nvfp4_quantize (or
+ * nvfp4_quantize_dual) made of it with the same `transposed`, `global_scale` and `sf_layout`,
+ *   sums[0] = sum (Q(x) - x)^2     sums[1] = sum x^2          (device doubles, overwritten)
+ * so that the paper's gradient-to-noise ratio ||x|| / (sigma_q sqrt(d)) = sqrt(sums[1] / sums[0]);
+ * the paper leaves FP4 for higher precision once this falls below sqrt(3).  One extra read of x and
+ * of the codes; sums is 8-byte aligned; other arguments and errors as for nvfp4_quantize.
+ */
+NVFP4_API int nvfp4_quantization_noise(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int transposed,
+                             const float* global_scale, const uint8_t* codes, const uint8_t* scales,
+                             int sf_layout, double* sums, void* cuda_stream);
+
 /* Per-tensor scale g = max|x| / (6*448), or 1.0f for an all-zero tensor, written
  * to *global_scale_out (device).  The paper defines only the block scale; this
  * optional factor keeps small-magnitude gradients inside the E4M3 scale range. */

@@ -48,6 +48,9 @@ def lib():
         L.nvfp4o_quantize_transposed.restype = None
         L.nvfp4o_quantize_transposed.argtypes = q
         L.nvfp4o_dequantize.restype = None
+        L.nvfp4o_noise_sums.restype = None
+        L.nvfp4o_noise_sums.argtypes = [_f32p, _u8p, _u8p, C.c_float, C.c_int64, C.c_int64,
+                                        np.ctypeslib.ndpointer(dtype=np.float64, flags="C_CONTIGUOUS")]
         L.nvfp4o_dequantize.argtypes = [_u8p, _u8p, C.c_float, C.c_int64, C.c_int64, _f32p]
         L.nvfp4o_tensor_amax_scale.restype = C.c_float
         L.nvfp4o_tensor_amax_scale.argtypes = [_f32p, C.c_int64]
@@ -151,6 +154,15 @@ def dequantize(codes, scales, g=1.0):
     lib().nvfp4o_dequantize(np.ascontiguousarray(codes), np.ascontiguousarray(scales),
                             float(np.float32(g)), Rq, half * 2, out)
     return out
+
+
+def noise_sums(x, codes, scales, g=1.0):
+    """(sum (Q(x)-x)^2, sum x^2) in double; x in the quantized orientation [Rq, Kq]."""
+    x = _f32(x)
+    out = np.zeros(2, dtype=np.float64)
+    lib().nvfp4o_noise_sums(x, np.ascontiguousarray(codes), np.ascontiguousarray(scales), float(np.float32(g)),
+                            x.shape[0], x.shape[1], out)
+    return float(out[0]), float(out[1])
 
 
 def tensor_amax_scale(x) -> float:

@@ -209,6 +209,26 @@ void nvfp4o_dequantize(const uint8_t* codes, const uint8_t* scales, float g,
     }
 }
 
+// Section 4: the quantization noise of a tensor against its own norm.  out[0] = sum (Q(x) - x)^2
+// (= d * sigma_q^2), out[1] = sum x^2 (= the squared norm); the paper's ratio |x| / (sigma_q sqrt(d))
+// is sqrt(out[1] / out[0]) and its threshold sqrt(3).
+void nvfp4o_noise_sums(const float* x, const uint8_t* codes, const uint8_t* scales, float g,
+                       int64_t Rq, int64_t Kq, double out[2]) {
+  const int64_t nkb = Kq / 16;
+  double err2 = 0.0, x2 = 0.0;
+  for (int64_t r = 0; r < Rq; ++r)
+    for (int64_t k = 0; k < Kq; ++k) {
+      uint8_t byte = codes[(r * Kq + k) / 2];
+      uint8_t nib = (k & 1) ? (byte >> 4) : (byte & 15);
+      float d = nvfp4o_e4m3_decode(scales[r * nkb + k / 16]) * g;
+      double e = (double)(code_value(nib) * d) - (double)x[r * Kq + k];
+      err2 += e * e;
+      x2 += (double)x[r * Kq + k] * (double)x[r * Kq + k];
+    }
+  out[0] = err2;
+  out[1] = x2;
+}
+
 float nvfp4o_tensor_amax_scale(const float* x, int64_t n) {
   float amax = 0.0f;
   for (int64_t i = 0; i < n; ++i) { float a = std::fabs(x[i]); if (a > amax) amax = a; }

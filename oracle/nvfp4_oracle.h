@@ -82,6 +82,12 @@ void nvfp4o_quantize_transposed(const float* x, int64_t rows, int64_t cols, floa
 void nvfp4o_dequantize(const uint8_t* codes, const uint8_t* scales, float g,
                        int64_t Rq, int64_t Kq, float* out);
 
+/* Section 4 (gradient-to-noise ratio): out[0] = sum over the tensor of (Q(x) - x)^2, out[1] = sum
+ * of x^2, in double; x in the quantized orientation [Rq, Kq], linear scales.  The paper's ratio
+ * ||x|| / (sigma_q sqrt(d)) is sqrt(out[1]/out[0]); it switches precision when that falls below sqrt(3). */
+void nvfp4o_noise_sums(const float* x, const uint8_t* codes, const uint8_t* scales, float g,
+                       int64_t Rq, int64_t Kq, double out[2]);
+
 /* g = amax / (6*448) in one fp32 division, 1.0f when amax == 0. */
 float nvfp4o_tensor_amax_scale(const float* x, int64_t n);
 

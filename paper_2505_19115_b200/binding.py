@@ -55,6 +55,8 @@ def lib():
     L.nvfp4_quantize.argtypes = [vp, ci, i64, i64, i64, ci, vp, rp, vp, vp, ci, vp]
     L.nvfp4_quantize_dual.restype = ci
     L.nvfp4_quantize_dual.argtypes = [vp, ci, i64, i64, i64, vp, rp, vp, vp, rp, vp, vp, ci, vp]
+    L.nvfp4_quantization_noise.restype = ci
+    L.nvfp4_quantization_noise.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, ci, vp, vp]
     L.nvfp4_tensor_amax_scale.restype = ci
     L.nvfp4_tensor_amax_scale.argtypes = [vp, ci, i64, i64, i64, vp, vp]
     L.nvfp4_gemm.restype = ci
@@ -158,6 +160,18 @@ def nvfp4_quantize_dual(x: torch.Tensor, global_scale: torch.Tensor = None, roun
                                    sf_layout, _stream(stream))
     _check(st, "nvfp4_quantize_dual")
     return cr, sr, ct, stt
+
+
+def nvfp4_quantization_noise(x: torch.Tensor, codes, scales, transposed: bool = False, global_scale=None,
+                             sf_layout: int = SF_LINEAR, stream=None) -> torch.Tensor:
+    """Device tensor of two doubles: sum (Q(x) - x)^2 and sum x^2 (Section 4's noise and norm)."""
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+    sums = torch.empty(2, dtype=torch.float64, device=x.device)
+    st = lib().nvfp4_quantization_noise(_ptr(x), _dtype_code(x), x.shape[0], x.shape[1], x.stride(0), int(transposed),
+                                        _ptr(global_scale), _ptr(codes), _ptr(scales), sf_layout, _ptr(sums),
+                                        _stream(stream))
+    _check(st, "nvfp4_quantization_noise")
+    return sums
 
 
 def nvfp4_tensor_amax_scale(x: torch.Tensor, out: torch.Tensor = None, stream=None) -> torch.Tensor:
