@@ -148,6 +148,22 @@ NVFP4_API int nvfp4_gemm(const uint8_t* a_codes, const uint8_t* a_sf, const floa
                int64_t M, int64_t N, int64_t K,
                void* d, int d_dtype, int64_t ldd, void* cuda_stream);
 
+/*
+ * The same product with the next quantization fused into the epilogue: instead of D, the call writes
+ * Q(D) with blocks of 16 along N (as nvfp4_quantize of the fp32 D with transposed == 0 would: codes
+ * [M, N/2], scales for the quantized shape (M, N) in `sf_layout`), so that a consumer which would
+ * quantize D along N anyway (the next layer's Q(X) of Eq. 4) never sees a high-precision copy.
+ * out_global_scale is the per-tensor scale of the OUTPUT (device, NULL => 1; it has to be known before
+ * the product runs: from the previous step, or a bound); rounding (host) as for nvfp4_quantize, the
+ * block index for SR being m*(N/16) + n/16.  The result equals nvfp4_quantize applied to the fp32
+ * output of nvfp4_gemm bit for bit.  N % 32 == 0, K % 32 == 0; alignment as for nvfp4_gemm.
+ */
+NVFP4_API int nvfp4_gemm_quantized(const uint8_t* a_codes, const uint8_t* a_sf, const float* a_g,
+                         const uint8_t* b_codes, const uint8_t* b_sf, const float* b_g,
+                         int64_t M, int64_t N, int64_t K,
+                         const float* out_global_scale, const nvfp4_rounding* rounding /* host */,
+                         uint8_t* out_codes, uint8_t* out_scales, int sf_layout, void* cuda_stream);
+
 /* Tuning/testing hook: force the GEMM kernel variant.  0 restores the automatic
  * choice; 128 / 256 select the single-CTA kernel with a 128 x {128,256} tile;
  * 2128 / 2192 / 2256 select the CTA-pair kernel with a 256 x {128,192,256} tile.

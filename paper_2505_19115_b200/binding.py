@@ -61,6 +61,8 @@ def lib():
     L.nvfp4_tensor_amax_scale.argtypes = [vp, ci, i64, i64, i64, vp, vp]
     L.nvfp4_gemm.restype = ci
     L.nvfp4_gemm.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, i64, vp]
+    L.nvfp4_gemm_quantized.restype = ci
+    L.nvfp4_gemm_quantized.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, rp, vp, vp, ci, vp]
     L.nvfp4_gemm_set_tile_n.restype = ci
     L.nvfp4_gemm_set_tile_n.argtypes = [ci]
     L.nvfp4_linear_workspace_bytes.restype = sz
@@ -195,6 +197,24 @@ def nvfp4_gemm(a_codes, a_sf, a_g, b_codes, b_sf, b_g, out_dtype=torch.float32, 
                           M, N, K, _ptr(out), _dtype_code(out), out.stride(0), _stream(stream))
     _check(st, "nvfp4_gemm")
     return out
+
+
+def nvfp4_gemm_quantized(a_codes, a_sf, a_g, b_codes, b_sf, b_g, out_global_scale=None, rounding: Rounding = None,
+                         sf_layout: int = SF_LINEAR, stream=None):
+    """Q(A . B^T) with blocks along N, straight from the GEMM epilogue.  Returns (codes [M, N/2], scales)."""
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    N = b_codes.shape[0]
+    rounding = rounding or Rounding()
+    codes = torch.empty((M, N // 2), dtype=torch.uint8, device=a_codes.device)
+    if sf_layout == SF_LINEAR:
+        scales = torch.empty((M, N // 16), dtype=torch.uint8, device=a_codes.device)
+    else:
+        scales = torch.empty(max(nvfp4_sf_bytes(M, N, sf_layout), 16), dtype=torch.uint8, device=a_codes.device)
+    st = lib().nvfp4_gemm_quantized(_ptr(a_codes), _ptr(a_sf), _ptr(a_g), _ptr(b_codes), _ptr(b_sf), _ptr(b_g), M, N, K,
+                                    _ptr(out_global_scale), C.byref(rounding), _ptr(codes), _ptr(scales), sf_layout,
+                                    _stream(stream))
+    _check(st, "nvfp4_gemm_quantized")
+    return codes, scales
 
 
 def nvfp4_gemm_set_tile_n(bn: int) -> None:

@@ -13,7 +13,7 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
-#include "common.cuh"
+#include "quantize_core.cuh"
 #include "tensor_map.cuh"
 
 namespace nvfp4 {
@@ -534,7 +534,7 @@ struct Cfg2 {
   static constexpr int kStageBytes = kABytes + kBBytes + kSfaBytes + kSfbBytes;
   static constexpr int kEpiWarpBytes = 2 * 4096;                   // two 32-row x 128-byte buffers per warp
   static constexpr int kEpiBytes = 4 * kEpiWarpBytes;
-  static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*align*/ + 512 /*barriers*/;
+  static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024 /*align*/ + 512 /*barriers*/ + 512 /*reciprocal table*/;
   // tensor memory: accumulators, then kSfBufs scale buffers of (16 columns for A, 16 per B tile)
   static constexpr uint32_t kSfaCol = kAccStages * BN;
   static constexpr uint32_t kSfCols = 16 + kSfbTiles * 16;
@@ -555,14 +555,25 @@ struct Gemm2Params {
   int M, N, K;
   int tiles_m, tiles_n, k_stages, k_tiles;
   int a_row_tiles, b_row_tiles;
+  // quantized output (OUT == 2): per-tensor scale of the output, rounding, scales destination
+  const float* out_g;
+  PhiloxStream out_rng;
+  uint8_t* out_scales;
+  int out_sr, out_swizzled;
+  int64_t out_nkb, out_k_tiles;
 };
 
-template <int BN, bool BF16_OUT>
+// OUT: 0 = fp32, 1 = bf16, 2 = the NVFP4 row quantization of the product (codes + scales), for a
+// consumer that would quantize D along N anyway (the next layer's Q(X) of Eq. 4): no high-precision
+// round trip through memory.
+template <int BN, int OUT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemm2Threads, 1)
 gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
                    const __grid_constant__ CUtensorMap map_d, const Gemm2Params p) {
   using C = Cfg2<BN>;
+  constexpr bool BF16_OUT = (OUT == 1), Q_OUT = (OUT == 2);
+  static_assert(!Q_OUT || BN == 256, "the quantized epilogue stores one 128-byte row of codes per tile row");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -581,6 +592,8 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   auto tempty_bar = [&](int a) { return bar_base + 8u * (3 * C::kStages + 2 * C::kSfBufs + C::kAccStages + a); };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * C::kNumBarriers);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  float* inv_table = reinterpret_cast<float*>(bar_gen + 512);   // OUT == 2 only: 1 / (decode(q) * out_g) per scale code
+  if constexpr (Q_OUT) build_inv_table(inv_table, p.out_g ? __ldg(p.out_g) : 1.0f);
 
   const int warp = __shfl_sync(0xFFFFFFFFu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();          // 0 = leader of the pair
@@ -774,6 +787,80 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
       tc_fence_after();
       const int row0 = tm * 256 + (int)rank * 128 + quarter * 32;
       const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
+      if constexpr (Q_OUT) {
+        // ---- quantized output: this lane's row, the tile's 256 columns = 16 blocks of 16 ----
+        const float cq = __fdiv_rn(__fdiv_rn(1.0f, 6.0f), p.out_g ? __ldg(p.out_g) : 1.0f);
+        const int64_t row = (int64_t)row0 + lane;
+        uint32_t codes[32];                          // 128 bytes of codes
+        uint32_t sfw[4] = {0u, 0u, 0u, 0u};          // 16 scale bytes, four per k-tile
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          uint32_t r[32];
+          tmem_ld32(t_row + 32 * c, r);
+          tmem_ld_wait();
+          tmem_ld_pin(r);
+          if (c == 7) {                              // accumulator fully read: hand it back to the leader
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(lead_tempty0 + 8u * acc);
+          }
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float v[16], amax = 0.0f;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              v[j] = __uint_as_float(r[16 * h + j]) * alpha;     // the value the fp32 epilogue would store
+              amax = fmaxf(amax, fabsf(v[j]));
+            }
+            const int kbl = 2 * c + h;
+            const uint64_t blk = (uint64_t)(row * p.out_nkb + (int64_t)tn * (BN / 16) + kbl);
+            uint32_t lo, hi, sf;
+            if (p.out_sr) encode_block<true>(v, amax, cq, inv_table, p.out_rng, blk, lo, hi, sf);
+            else encode_block<false>(v, amax, cq, inv_table, p.out_rng, blk, lo, hi, sf);
+            codes[2 * kbl] = lo;
+            codes[2 * kbl + 1] = hi;
+            sfw[kbl >> 2] |= sf << (8 * (kbl & 3));
+          }
+        }
+        // codes: stage 32 rows x 128 bytes (128-byte swizzle) and store them as one box
+        const uint32_t buf = my_buf + (chunk_no & 1u) * 4096u;
+        if (chunk_no >= 2) {
+          if (lane == 0) tma_store_wait_read<1>();
+          __syncwarp();
+        }
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint32_t dst = buf + lane * 128 + ((c ^ (lane & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(codes[4 * c]), "r"(codes[4 * c + 1]),
+                       "r"(codes[4 * c + 2]), "r"(codes[4 * c + 3]) : "memory");
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_2d(&map_d, buf, tn * (BN / 2), row0);
+          tma_store_commit();
+        }
+        ++chunk_no;
+        // scales
+        if (p.out_swizzled) {
+          if ((row >> 7) < (((int64_t)p.M + 127) >> 7)) {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              const int64_t kt = (int64_t)tn * (BN / 64) + t;
+              if (kt < p.out_k_tiles)
+                *reinterpret_cast<uint32_t*>(p.out_scales + sf_swizzled_offset(row, kt * 4, p.out_k_tiles)) = sfw[t];
+            }
+          }
+        } else if (row < p.M) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int64_t kb = (int64_t)tn * (BN / 16) + i;
+            if (kb < p.out_nkb) p.out_scales[row * p.out_nkb + kb] = (uint8_t)(sfw[i >> 2] >> (8 * (i & 3)));
+          }
+        }
+        if (++acc == C::kAccStages) { acc = 0; acc_ph ^= 1u; }
+        continue;
+      }
       // The MMA issuer cannot start the next tile before this accumulator is read out, so the read-out is
       // what must finish early, not the stores: the first kHeld chunks are converted and parked in
       // registers, the others stream through the staging buffers, the accumulator is handed back
@@ -928,24 +1015,54 @@ int launch_gemm(const uint8_t* a_codes, const uint8_t* b_codes, GemmParams p, cu
   return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
-template <int BN, bool BF16_OUT>
-int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParams& g, cudaStream_t s) {
+// Output of the quantized epilogue (OUT == 2); unused otherwise.
+struct QuantOut {
+  const float* g = nullptr;
+  const nvfp4_rounding* rounding = nullptr;
+  uint8_t* codes = nullptr;
+  uint8_t* scales = nullptr;
+  int sf_layout = NVFP4_SF_LINEAR;
+};
+
+// Packed codes of the quantized output [M, N/2 bytes] -> boxes of 32 rows x 128 bytes, 128-byte swizzle.
+bool make_qout_map(CUtensorMap* map, uint8_t* base, int64_t M, int64_t N) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)(N / 2), (cuuint64_t)M};
+  const cuuint64_t strides[1] = {(cuuint64_t)(N / 2)};
+  const cuuint32_t box[2] = {128, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int OUT>
+int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParams& g, cudaStream_t s,
+                 const QuantOut& q = QuantOut()) {
   using C = Cfg2<BN>;
   CUtensorMap map_a, map_b, map_sfa, map_sfb, map_d;
   if (!make_codes_map(&map_a, a_codes, g.M, g.K / 2, 128)) return NVFP4_ERR_CUDA;
   if (!make_codes_map(&map_b, b_codes, g.N, g.K / 2, BN / 2)) return NVFP4_ERR_CUDA;
   if (!make_sf_map(&map_sfa, g.a_sf, (int64_t)g.a_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
   if (!make_sf_map(&map_sfb, g.b_sf, (int64_t)g.b_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
-  if (!make_out_map(&map_d, g.d, g.M, g.N, g.ldd, BF16_OUT)) return NVFP4_ERR_CUDA;
+  if constexpr (OUT == 2) {
+    if (!make_qout_map(&map_d, q.codes, g.M, g.N)) return NVFP4_ERR_CUDA;
+  } else {
+    if (!make_out_map(&map_d, g.d, g.M, g.N, g.ldd, OUT == 1)) return NVFP4_ERR_CUDA;
+  }
   Gemm2Params p;
   p.a_g = g.a_g; p.b_g = g.b_g; p.M = g.M; p.N = g.N; p.K = g.K;
   p.tiles_m = (g.M + 255) / 256;
   p.tiles_n = (g.N + BN - 1) / BN;
   p.k_stages = g.k_stages; p.k_tiles = g.k_tiles;
   p.a_row_tiles = g.a_row_tiles; p.b_row_tiles = g.b_row_tiles;
+  p.out_g = q.g; p.out_scales = q.scales; p.out_sr = 0; p.out_swizzled = q.sf_layout == NVFP4_SF_SWIZZLED_128x4;
+  p.out_nkb = g.N / 16; p.out_k_tiles = ceil_div(p.out_nkb, 4);
+  philox_stream_init(&p.out_rng, q.rounding ? q.rounding->seed : 0, q.rounding ? q.rounding->offset : 0);
+  if (q.rounding) p.out_sr = q.rounding->mode == NVFP4_SR;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm2_nvfp4_kernel<BN, BF16_OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(gemm2_nvfp4_kernel<BN, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::kSmemBytes) != cudaSuccess)
       return NVFP4_ERR_CUDA;
     attr_set = true;
@@ -953,13 +1070,13 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
   const int tiles = p.tiles_m * p.tiles_n;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  gemm2_nvfp4_kernel<BN, BF16_OUT><<<2 * pairs, kGemm2Threads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
+  gemm2_nvfp4_kernel<BN, OUT><<<2 * pairs, kGemm2Threads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
   return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
 template <int BN>
 int launch_gemm2_dt(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParams& g, cudaStream_t s) {
-  return g.d_is_bf16 ? launch_gemm2<BN, true>(a_codes, b_codes, g, s) : launch_gemm2<BN, false>(a_codes, b_codes, g, s);
+  return g.d_is_bf16 ? launch_gemm2<BN, 1>(a_codes, b_codes, g, s) : launch_gemm2<BN, 0>(a_codes, b_codes, g, s);
 }
 
 }  // namespace
@@ -1011,6 +1128,34 @@ extern "C" int nvfp4_gemm(const uint8_t* a_codes, const uint8_t* a_sf, const flo
     case 2192: return launch_gemm2_dt<192>(a_codes, b_codes, p, s);
     default: return launch_gemm2_dt<256>(a_codes, b_codes, p, s);
   }
+}
+
+extern "C" int nvfp4_gemm_quantized(const uint8_t* a_codes, const uint8_t* a_sf, const float* a_g,
+                                    const uint8_t* b_codes, const uint8_t* b_sf, const float* b_g,
+                                    int64_t M, int64_t N, int64_t K,
+                                    const float* out_global_scale, const nvfp4_rounding* rounding,
+                                    uint8_t* out_codes, uint8_t* out_scales, int sf_layout, void* cuda_stream) {
+  if (!a_codes || !a_sf || !b_codes || !b_sf || !rounding || !out_codes || !out_scales) return NVFP4_ERR_NULL;
+  if ((rounding->mode != NVFP4_RTN && rounding->mode != NVFP4_SR) || rounding->reserved != 0) return NVFP4_ERR_ENUM;
+  if (sf_layout != NVFP4_SF_LINEAR && sf_layout != NVFP4_SF_SWIZZLED_128x4) return NVFP4_ERR_ENUM;
+  if (M <= 0 || N <= 0 || K <= 0 || (K % 32) != 0 || (N % 32) != 0) return NVFP4_ERR_SHAPE;
+  if (M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256 || K >= (1ll << 31) - 256) return NVFP4_ERR_SHAPE;
+  if (!aligned16(a_codes) || !aligned16(a_sf) || !aligned16(b_codes) || !aligned16(b_sf) || !aligned16(out_codes) ||
+      !aligned16(out_scales))
+    return NVFP4_ERR_ALIGN;
+  if (int st = check_arch()) return st;
+  GemmParams p;
+  p.a_sf = a_sf; p.b_sf = b_sf; p.a_g = a_g; p.b_g = b_g; p.d = nullptr; p.ldd = N;
+  p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  p.k_stages = (int)ceil_div(K, BK);
+  p.k_tiles = (int)ceil_div(K, MMA_K);
+  p.a_row_tiles = (int)ceil_div(M, 128);
+  p.b_row_tiles = (int)ceil_div(N, 128);
+  p.d_is_bf16 = 0;
+  p.tiles_m = p.tiles_n = 0;
+  QuantOut q;
+  q.g = out_global_scale; q.rounding = rounding; q.codes = out_codes; q.scales = out_scales; q.sf_layout = sf_layout;
+  return launch_gemm2<256, 2>(a_codes, b_codes, p, static_cast<cudaStream_t>(cuda_stream), q);
 }
 
 extern "C" int nvfp4_device_error_word(uint32_t* host_out) {

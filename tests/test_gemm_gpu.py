@@ -123,3 +123,30 @@ def test_many_tiles_persistent_schedule():
     ref, T = ob.gemm_sampled(*ora_ops, ii, jj)
     got = D.cpu().numpy()[ii, jj]
     assert np.all(np.abs(got - ref) <= TOL * T)
+
+
+# ---------------------------------------------------------------- quantization fused into the epilogue
+@pytest.mark.parametrize("sf_layout", [nb.SF_LINEAR, nb.SF_SWIZZLED])
+@pytest.mark.parametrize("mode", [nb.RTN, nb.SR])
+@pytest.mark.parametrize("shape", [(256, 256, 256), (300, 544, 512), (1000, 1312, 1056), (64, 32, 64)])
+def test_quantized_epilogue_equals_quantizing_the_fp32_product(shape, mode, sf_layout):
+    M, N, K = shape
+    gpu_ops, ora_ops = _quantized_pair(M, N, K, seed=90 + M)
+    D = nb.nvfp4_gemm(*gpu_ops)
+    g_out = nb.nvfp4_tensor_amax_scale(D)
+    r = nb.Rounding(mode, 17, 3)
+    want_c, want_s = nb.nvfp4_quantize(D, False, g_out, r, sf_layout)
+    got_c, got_s = nb.nvfp4_gemm_quantized(*gpu_ops, out_global_scale=g_out, rounding=r, sf_layout=sf_layout)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
+    assert torch.equal(got_c, want_c)
+    assert torch.equal(got_s.reshape(-1), want_s.reshape(-1))
+    if sf_layout == nb.SF_LINEAR:
+        # against the oracle's product: every dequantized output within one grid step (two under SR) of it
+        ref, T = ob.gemm(*ora_ops)
+        g = float(g_out.item())
+        deq = ob.dequantize(got_c.cpu().numpy(), got_s.cpu().numpy(), g)
+        step = np.repeat(np.array([ob.e4m3_decode(int(b)) for b in got_s.cpu().numpy().reshape(-1)],
+                                  dtype=np.float64).reshape(M, N // 16), 16, axis=1) * g * 2.0
+        slack = (1.0 if mode == nb.RTN else 2.0) * step + TOL * T      # also covers the clip of a block's maximum at 6
+        assert np.all(np.abs(deq - ref) <= slack)
