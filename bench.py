@@ -22,7 +22,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2505_19115_b200 import synth  # noqa: E402
+from paper_2505_19115_b200 import replicas, synth  # noqa: E402
 
 METRIC = "NVFP4 linear fwd+bwd TFLOPS (% FP4 peak); quantizer GB/s (% HBM peak)"
 FP4_OVER_BF16 = 4.0        # nominal dense ratio: 9 PFLOP/s NVFP4 vs 2.25 PFLOP/s bf16
@@ -180,9 +180,7 @@ def main():
 
     from paper_2505_19115_b200 import binding as nb
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = replicas.env_rank_world()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     dist = None
@@ -199,7 +197,7 @@ def main():
     # ---- resident inputs: every rank has its own block (replicas; no data-path collective) ----
     layers = []
     for li, (name, K, N) in enumerate(cfg["linears"]):
-        X, W, dY = synth.linear_inputs(M, K, N, seed=4000 + 10 * li + 100 * rank, device=dev)
+        X, W, dY = synth.linear_inputs(M, K, N, seed=replicas.replica_seed(4000 + 10 * li, rank), device=dev)
         layers.append(dict(name=name, K=K, N=N, X=X, W=W, dY=dY,
                            Y=torch.empty((M, N), dtype=torch.float32, device=dev),
                            dX=torch.empty((M, K), dtype=torch.float32, device=dev),
@@ -249,14 +247,11 @@ def main():
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     ms = e0.elapsed_time(e1)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = replicas.max_over_ranks(ms, dist, dev)
     err_word = nb.nvfp4_device_error_word()
     if err_word:
         raise RuntimeError(f"device error word {err_word:#x}: a kernel gave up on a bounded wait")
-    value = flops_per_step * args.steps * world / (ms * 1e-3) / 1e12
+    value = replicas.aggregate_throughput(flops_per_step * args.steps, world, ms * 1e-3) / 1e12
 
     # ---- roofline of the dominant kernel (the GEMM): same workload, decomposed into the C-ABI's
     #      quantize and gemm calls so that CUDA events bracket every GEMM launch ----
@@ -420,10 +415,7 @@ def main():
         f1.record()
         barrier()
         ems = f0.elapsed_time(f1)
-        if dist is not None:
-            t = torch.tensor([ems], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
+        ems = replicas.max_over_ranks(ems, dist, dev)
         e2e = {"value": flops_per_step * e2e_steps * world / (ems * 1e-3) / 1e12, "unit": "TFLOPS",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
                "ms_per_step": ems / e2e_steps}
