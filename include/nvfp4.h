@@ -245,6 +245,26 @@ NVFP4_API int nvfp4_linear_bwd(const void* dY, const void* W, const void* X, int
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Quantization-aware fine-tuning phase (Section 5): the forward pass stays in NVFP4
+ * (nvfp4_linear_fwd), the backward and update products run in BF16.
+ *
+ * nvfp4_gemm_bf16: D[M,N] = A[M,K] . B[N,K]^T for dense bf16 A and B (both contiguous along K),
+ * fp32 accumulation, D fp32 or bf16 with leading dimension ldd.  K % 16 == 0, pointers 16-byte
+ * aligned, ldd*sizeof(D) a multiple of 16.
+ * nvfp4_transpose_bf16: out[cols, rows] = x[rows, cols]^T (rows, cols multiples of 8; out dense).
+ * nvfp4_linear_bwd_bf16: dX[M,K] = dY . W and dW[N,K] = dY^T . X from bf16 dY[M,N], W[N,K], X[M,K]
+ * (all dense): transposes W, X and dY into the workspace (nvfp4_linear_bwd_bf16_workspace_bytes,
+ * 256-byte aligned) and runs the two products.  M, N, K multiples of 16.
+ */
+NVFP4_API int nvfp4_gemm_bf16(const void* a, const void* b, int64_t M, int64_t N, int64_t K,
+                    void* d, int d_dtype, int64_t ldd, void* cuda_stream);
+NVFP4_API int nvfp4_transpose_bf16(const void* x, int64_t rows, int64_t cols, int64_t ld, void* out, void* cuda_stream);
+NVFP4_API size_t nvfp4_linear_bwd_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K);
+NVFP4_API int nvfp4_linear_bwd_bf16(const void* dY, const void* W, const void* X, int64_t M, int64_t N, int64_t K,
+                          void* dX, int dx_dtype, void* dW, int dw_dtype,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * nvfp4_linear_fwd without a caller-supplied workspace and without any device-memory
  * allocation (the paper has no counterpart; this is a library convenience).
  *

@@ -48,6 +48,8 @@ def lib():
         L.nvfp4o_quantize_transposed.restype = None
         L.nvfp4o_quantize_transposed.argtypes = q
         L.nvfp4o_dequantize.restype = None
+        L.nvfp4o_matmul_nt.restype = None
+        L.nvfp4o_matmul_nt.argtypes = [_f32p, _f32p, C.c_int64, C.c_int64, C.c_int64, _f32p, _f32p, C.c_int]
         L.nvfp4o_noise_sums.restype = None
         L.nvfp4o_noise_sums.argtypes = [_f32p, _u8p, _u8p, C.c_float, C.c_int64, C.c_int64,
                                         np.ctypeslib.ndpointer(dtype=np.float64, flags="C_CONTIGUOUS")]
@@ -163,6 +165,17 @@ def noise_sums(x, codes, scales, g=1.0):
     lib().nvfp4o_noise_sums(x, np.ascontiguousarray(codes), np.ascontiguousarray(scales), float(np.float32(g)),
                             x.shape[0], x.shape[1], out)
     return float(out[0]), float(out[1])
+
+
+def matmul_nt(A, B, nthreads=None):
+    """(A . B^T rounded to fp32 from a double accumulation, sum |a b|) for plain fp32 arrays A[M,K], B[N,K]."""
+    A, B = _f32(A), _f32(B)
+    M, K = A.shape
+    N = B.shape[0]
+    D = np.zeros((M, N), dtype=np.float32)
+    T = np.zeros((M, N), dtype=np.float32)
+    lib().nvfp4o_matmul_nt(A, B, M, N, K, D, T, host_threads() if nthreads is None else nthreads)
+    return D, T
 
 
 def tensor_amax_scale(x) -> float:

@@ -229,6 +229,24 @@ void nvfp4o_noise_sums(const float* x, const uint8_t* codes, const uint8_t* scal
   out[1] = x2;
 }
 
+// QAF phase (Section 5): backward and update GEMMs on unquantized (bf16) operands.
+// D[i,j] = sum_k A[i,k] * B[j,k] in double, rounded to fp32; T = the same sum over absolute values.
+void nvfp4o_matmul_nt(const float* A, const float* B, int64_t M, int64_t N, int64_t K, float* D, float* T, int nthreads) {
+  parallel_rows(M, nthreads, [=](int64_t r0, int64_t r1) {
+    for (int64_t i = r0; i < r1; ++i)
+      for (int64_t j = 0; j < N; ++j) {
+        double acc = 0.0, aabs = 0.0;
+        for (int64_t k = 0; k < K; ++k) {
+          double pr = (double)A[i * K + k] * (double)B[j * K + k];
+          acc += pr;
+          aabs += std::fabs(pr);
+        }
+        if (D) D[i * N + j] = (float)acc;
+        if (T) T[i * N + j] = (float)aabs;
+      }
+  });
+}
+
 float nvfp4o_tensor_amax_scale(const float* x, int64_t n) {
   float amax = 0.0f;
   for (int64_t i = 0; i < n; ++i) { float a = std::fabs(x[i]); if (a > amax) amax = a; }

@@ -88,6 +88,10 @@ void nvfp4o_dequantize(const uint8_t* codes, const uint8_t* scales, float g,
 void nvfp4o_noise_sums(const float* x, const uint8_t* codes, const uint8_t* scales, float g,
                        int64_t Rq, int64_t Kq, double out[2]);
 
+/* QAF phase (Section 5: forward FP4, backward and update BF16): D = A[M,K] . B[N,K]^T on plain
+ * (unquantized) operands, double accumulation, rounded to fp32; T = sum |a_k b_k|. */
+void nvfp4o_matmul_nt(const float* A, const float* B, int64_t M, int64_t N, int64_t K, float* D, float* T, int nthreads);
+
 /* g = amax / (6*448) in one fp32 division, 1.0f when amax == 0. */
 float nvfp4o_tensor_amax_scale(const float* x, int64_t n);
 

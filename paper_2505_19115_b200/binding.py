@@ -81,6 +81,14 @@ def lib():
     L.nvfp4_linear_bwd_saved.argtypes = [vp, ci, i64, i64, i64, ci, vp, rp, rp, vp, sz, vp, ci, vp, ci, vp, sz, vp]
     L.nvfp4_linear_bwd.restype = ci
     L.nvfp4_linear_bwd.argtypes = [vp, vp, vp, ci, i64, i64, i64, ci, vp, vp, vp, rp, rp, rp, rp, vp, ci, vp, ci, vp, sz, vp]
+    L.nvfp4_gemm_bf16.restype = ci
+    L.nvfp4_gemm_bf16.argtypes = [vp, vp, i64, i64, i64, vp, ci, i64, vp]
+    L.nvfp4_transpose_bf16.restype = ci
+    L.nvfp4_transpose_bf16.argtypes = [vp, i64, i64, i64, vp, vp]
+    L.nvfp4_linear_bwd_bf16_workspace_bytes.restype = sz
+    L.nvfp4_linear_bwd_bf16_workspace_bytes.argtypes = [i64, i64, i64]
+    L.nvfp4_linear_bwd_bf16.restype = ci
+    L.nvfp4_linear_bwd_bf16.argtypes = [vp, vp, vp, i64, i64, i64, vp, ci, vp, ci, vp, sz, vp]
     L.nvfp4_linear_fwd_static.restype = ci
     L.nvfp4_linear_fwd_static.argtypes = [vp, vp, ci, i64, i64, i64, ci, vp, vp, rp, rp, vp, ci, vp]
     L.nvfp4_device_error_word.restype = ci
@@ -328,6 +336,36 @@ def nvfp4_linear_bwd(dY, W, X, gscale_mode=G_AMAX, gdy=None, gw=None, gx=None, r
                                 C.byref(rwt or Rounding(RTN)), C.byref(rxt or Rounding(SR, 0, 2)),
                                 _ptr(dX), _dtype_code(dX), _ptr(dW), _dtype_code(dW), _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "nvfp4_linear_bwd")
+    return dX, dW
+
+
+def nvfp4_gemm_bf16(A, B, out_dtype=torch.float32, out=None, stream=None):
+    """D[M,N] = A[M,K] . B[N,K]^T on bf16 operands (the QAF phase's backward / update precision)."""
+    assert A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and A.is_contiguous() and B.is_contiguous()
+    (M, K), N = A.shape, B.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=A.device)
+    _check(lib().nvfp4_gemm_bf16(_ptr(A), _ptr(B), M, N, K, _ptr(out), _dtype_code(out), out.stride(0), _stream(stream)),
+           "nvfp4_gemm_bf16")
+    return out
+
+
+def nvfp4_transpose_bf16(x, stream=None):
+    assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1
+    out = torch.empty((x.shape[1], x.shape[0]), dtype=torch.bfloat16, device=x.device)
+    _check(lib().nvfp4_transpose_bf16(_ptr(x), x.shape[0], x.shape[1], x.stride(0), _ptr(out), _stream(stream)),
+           "nvfp4_transpose_bf16")
+    return out
+
+
+def nvfp4_linear_bwd_bf16(dY, W, X, dx_dtype=torch.float32, dw_dtype=torch.float32, workspace=None, stream=None):
+    """QAF backward + update in BF16: returns (dX[M,K], dW[N,K])."""
+    (M, N), K = dY.shape, W.shape[1]
+    dX = torch.empty((M, K), dtype=dx_dtype, device=dY.device)
+    dW = torch.empty((N, K), dtype=dw_dtype, device=dY.device)
+    ws = _scratch(int(lib().nvfp4_linear_bwd_bf16_workspace_bytes(M, N, K)), dY.device, workspace)
+    _check(lib().nvfp4_linear_bwd_bf16(_ptr(dY), _ptr(W), _ptr(X), M, N, K, _ptr(dX), _dtype_code(dX), _ptr(dW),
+                                       _dtype_code(dW), _ptr(ws), ws.numel(), _stream(stream)), "nvfp4_linear_bwd_bf16")
     return dX, dW
 
 

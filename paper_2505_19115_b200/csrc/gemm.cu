@@ -287,6 +287,16 @@ __device__ __forceinline__ void tc_mma_nvf4_pair(uint32_t d_tmem, uint64_t adesc
                : "memory");
 }
 
+// bf16 x bf16 -> fp32, 256 x N x 16 per instruction (the backward / update products of the paper's
+// quantization-aware fine-tuning phase, which run in BF16)
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\t"
+               "setp.ne.b32 p, %4, 0;\n\t"
+               "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
 // Shared-memory matrix descriptors (64-bit): start address, leading/stride byte offsets (all >> 4),
 // descriptor version 1 at bit 46, swizzle mode at bits 61-63.
 // Operand tiles: K-major, 128-byte swizzle, rows 128 bytes apart, 8-row groups 1024 bytes apart.
@@ -300,6 +310,10 @@ __device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
 }
 // Instruction descriptor of kind::mxf4nvf4: E2M1 x E2M1 (format 1), K-major operands, UE4M3
 // scales, N >> 3 at bit 17, M >> 4 at bit 24.
+// Instruction descriptor of kind::f16 with bf16 operands (format 1) and an fp32 accumulator (bit 4).
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
 __host__ __device__ constexpr uint32_t instr_desc(int m, int n) {
   return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (0u << 23) | ((uint32_t)(m >> 4) << 24);
 }
@@ -566,7 +580,9 @@ struct Gemm2Params {
 // OUT: 0 = fp32, 1 = bf16, 2 = the NVFP4 row quantization of the product (codes + scales), for a
 // consumer that would quantize D along N anyway (the next layer's Q(X) of Eq. 4): no high-precision
 // round trip through memory.
-template <int BN, int OUT>
+// BF16_IN: operands are plain bf16 [rows, K] (K-major) instead of packed codes with scales; the scale
+// producer and the scale movers then have nothing to do and a k-stage is 64 values (128 bytes per row).
+template <int BN, int OUT, bool BF16_IN = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemm2Threads, 1)
 gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
@@ -647,12 +663,12 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     }
   } else if (warp == 10) {
     // ------------------------------- scale producer (both CTAs) -------------------------------
-    const bool issuer = elect_one();
+    const bool issuer = elect_one() && !BF16_IN;
     int s = 0;
     uint32_t ph = 0;
     bool ok = true;
     constexpr uint32_t kScaleTx = C::kSfaBytes + C::kSfbBytes;     // signalled on this CTA's own barrier
-    for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+    for (int tile = pair; !BF16_IN && ok && tile < num_tiles; tile += num_pairs) {
       int tm, tn;
       tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
       const int a_row = min(tm * 2 + (int)rank, p.a_row_tiles - 1) * p.k_tiles;
@@ -681,7 +697,7 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     // ------------------------------- MMA issuer (leader CTA only) -------------------------------
     if (rank == 0) {
       const bool issuer = elect_one();
-      constexpr uint32_t idesc = instr_desc(256, BN);
+      constexpr uint32_t idesc = BF16_IN ? instr_desc_bf16(256, BN) : instr_desc(256, BN);
       int s = 0, b = 0, acc = 0;
       uint32_t ph = 0, bph = 0, acc_ph = 0;
       bool ok = true;
@@ -693,14 +709,19 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int ks = 0; ks < p.k_stages; ++ks) {
           if (!(ok = mbar_wait_issuer(full_bar(s), ph, abort_flag, 0x13))) break;
-          if (!(ok = mbar_wait_issuer(sfr_bar(b), bph, abort_flag, 0x15))) break;
+          if constexpr (!BF16_IN) {
+            if (!(ok = mbar_wait_issuer(sfr_bar(b), bph, abort_flag, 0x15))) break;
+          }
           tc_fence_after();
           const uint32_t st = smem_base + s * C::kStageBytes;
           const int nkt = min(4, p.k_tiles - ks * 4);
           const uint32_t sfa_t = tmem_base + C::kSfaCol + b * C::kSfCols;
           const uint32_t sfb_t = sfa_t + 16 + sfb_off;
           const uint64_t adesc = operand_desc(st), bdesc = operand_desc(st + C::kABytes);
-          if (issuer) {
+          if (issuer && BF16_IN) {
+            for (int j = 0; j < nkt; ++j) tc_mma_bf16_pair(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, (ks | j) ? 1u : 0u);
+            tc_commit_pair(empty_bar(s));
+          } else if (issuer) {
             if (nkt == 4) {
 #pragma unroll
               for (int j = 0; j < 4; ++j)
@@ -732,7 +753,7 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     int s = 0, b = 0;
     uint32_t ph = 0, bph = 0;
     bool ok = true;
-    for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+    for (int tile = pair; !BF16_IN && ok && tile < num_tiles; tile += num_pairs) {
       for (int ks = 0; ks < p.k_stages; ++ks) {
         if (!(ok = mbar_wait_warp(sfl_bar(s), ph, abort_flag, 0x16))) break;
         if constexpr (!C::kSfFollowsStage) {        // otherwise buffer b == stage s, free once sfl_bar(s) could be armed
@@ -1036,15 +1057,21 @@ bool make_qout_map(CUtensorMap* map, uint8_t* base, int64_t M, int64_t N) {
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int OUT>
+template <int BN, int OUT, bool BF16_IN = false>
 int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParams& g, cudaStream_t s,
                  const QuantOut& q = QuantOut()) {
   using C = Cfg2<BN>;
   CUtensorMap map_a, map_b, map_sfa, map_sfb, map_d;
-  if (!make_codes_map(&map_a, a_codes, g.M, g.K / 2, 128)) return NVFP4_ERR_CUDA;
-  if (!make_codes_map(&map_b, b_codes, g.N, g.K / 2, BN / 2)) return NVFP4_ERR_CUDA;
-  if (!make_sf_map(&map_sfa, g.a_sf, (int64_t)g.a_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
-  if (!make_sf_map(&map_sfb, g.b_sf, (int64_t)g.b_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
+  const int64_t row_bytes = BF16_IN ? (int64_t)g.K * 2 : g.K / 2;       // operand rows as bytes
+  if (!make_codes_map(&map_a, a_codes, g.M, row_bytes, 128)) return NVFP4_ERR_CUDA;
+  if (!make_codes_map(&map_b, b_codes, g.N, row_bytes, BN / 2)) return NVFP4_ERR_CUDA;
+  if constexpr (BF16_IN) {
+    map_sfa = map_a;                                                     // never used by the kernel
+    map_sfb = map_b;
+  } else {
+    if (!make_sf_map(&map_sfa, g.a_sf, (int64_t)g.a_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
+    if (!make_sf_map(&map_sfb, g.b_sf, (int64_t)g.b_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
+  }
   if constexpr (OUT == 2) {
     if (!make_qout_map(&map_d, q.codes, g.M, g.N)) return NVFP4_ERR_CUDA;
   } else {
@@ -1062,7 +1089,7 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
   if (q.rounding) p.out_sr = q.rounding->mode == NVFP4_SR;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm2_nvfp4_kernel<BN, OUT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(gemm2_nvfp4_kernel<BN, OUT, BF16_IN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::kSmemBytes) != cudaSuccess)
       return NVFP4_ERR_CUDA;
     attr_set = true;
@@ -1070,7 +1097,7 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
   const int tiles = p.tiles_m * p.tiles_n;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  gemm2_nvfp4_kernel<BN, OUT><<<2 * pairs, kGemm2Threads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
+  gemm2_nvfp4_kernel<BN, OUT, BF16_IN><<<2 * pairs, kGemm2Threads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
   return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
@@ -1156,6 +1183,30 @@ extern "C" int nvfp4_gemm_quantized(const uint8_t* a_codes, const uint8_t* a_sf,
   QuantOut q;
   q.g = out_global_scale; q.rounding = rounding; q.codes = out_codes; q.scales = out_scales; q.sf_layout = sf_layout;
   return launch_gemm2<256, 2>(a_codes, b_codes, p, static_cast<cudaStream_t>(cuda_stream), q);
+}
+
+extern "C" int nvfp4_gemm_bf16(const void* a, const void* b, int64_t M, int64_t N, int64_t K,
+                               void* d, int d_dtype, int64_t ldd, void* cuda_stream) {
+  if (!a || !b || !d) return NVFP4_ERR_NULL;
+  if (d_dtype != NVFP4_BF16 && d_dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || ldd < N) return NVFP4_ERR_SHAPE;
+  if (M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256 || K >= (1ll << 30)) return NVFP4_ERR_SHAPE;
+  const int64_t esz = (d_dtype == NVFP4_BF16) ? 2 : 4;
+  if (!aligned16(a) || !aligned16(b) || !aligned16(d) || ((ldd * esz) % 16) != 0) return NVFP4_ERR_ALIGN;
+  if (int st = check_arch()) return st;
+  GemmParams p;
+  p.a_sf = p.b_sf = nullptr; p.a_g = p.b_g = nullptr; p.d = d; p.ldd = ldd;
+  p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  p.k_stages = (int)ceil_div(K * 2, BK_BYTES);       // 64 bf16 values per stage
+  p.k_tiles = (int)(K / 16);                         // 32-byte steps = one MMA each
+  p.a_row_tiles = (int)ceil_div(M, 128);
+  p.b_row_tiles = (int)ceil_div(N, 128);
+  p.d_is_bf16 = (d_dtype == NVFP4_BF16);
+  p.tiles_m = p.tiles_n = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const uint8_t* ab = static_cast<const uint8_t*>(a);
+  const uint8_t* bb = static_cast<const uint8_t*>(b);
+  return p.d_is_bf16 ? launch_gemm2<256, 1, true>(ab, bb, p, s) : launch_gemm2<256, 0, true>(ab, bb, p, s);
 }
 
 extern "C" int nvfp4_device_error_word(uint32_t* host_out) {

@@ -30,7 +30,7 @@ def _time(fn, iters, warmup):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("kernel", choices=["gemm", "quantize", "dual", "amax"])
+    ap.add_argument("kernel", choices=["gemm", "gemm_bf16", "transpose", "quantize", "dual", "amax"])
     ap.add_argument("--m", type=int, default=8192)
     ap.add_argument("--n", type=int, default=8192)
     ap.add_argument("--k", type=int, default=4096)
@@ -61,6 +61,17 @@ def main():
         flops = 2.0 * a.m * a.n * a.k
         res = {"kernel": "gemm", "m": a.m, "n": a.n, "k": a.k, "tile_n": a.tile_n, "out": str(out.dtype),
                "ms": ms, "TFLOP/s": flops / ms / 1e9}
+    elif a.kernel == "gemm_bf16":
+        A = synth.normal((a.m, a.k), 1.0, 1, device=dev)
+        B = synth.normal((a.n, a.k), 0.02, 2, device=dev)
+        out = torch.empty((a.m, a.n), dtype=torch.bfloat16 if a.bf16_out else torch.float32, device=dev)
+        ms = _time(lambda: nb.nvfp4_gemm_bf16(A, B, out=out), a.iters, a.warmup)
+        res = {"kernel": "gemm_bf16", "m": a.m, "n": a.n, "k": a.k, "out": str(out.dtype), "ms": ms,
+               "TFLOP/s": 2.0 * a.m * a.n * a.k / ms / 1e9}
+    elif a.kernel == "transpose":
+        x = synth.normal((a.rows, a.cols), 1.0, 3, device=dev)
+        ms = _time(lambda: nb.nvfp4_transpose_bf16(x), a.iters, a.warmup)
+        res = {"kernel": "transpose", "rows": a.rows, "cols": a.cols, "ms": ms, "GB/s": a.rows * a.cols * 4 / ms / 1e6}
     elif a.kernel == "quantize":
         dt = torch.float32 if a.fp32 else torch.bfloat16
         x = synth.heavy_tailed((a.rows, a.cols), 1002, device=dev, dtype=dt)

@@ -404,6 +404,19 @@ def test_noise_sums_against_numpy_and_the_uniform_noise_closed_form():
         assert abs(e2 / n - want) < 0.01 * want * 3
 
 
+def test_matmul_nt_against_float64_library_matmul():
+    rng = np.random.default_rng(31)
+    A = rng.standard_normal((37, 96)).astype(np.float32)
+    B = rng.standard_normal((21, 96)).astype(np.float32)
+    D, T = ob.matmul_nt(A, B, nthreads=3)
+    ref = A.astype(np.float64) @ B.astype(np.float64).T
+    assert np.array_equal(D, ref.astype(np.float32)) or np.max(np.abs(D - ref)) <= 1e-6 * np.max(np.abs(ref))
+    assert np.allclose(T, np.abs(A).astype(np.float64) @ np.abs(B).astype(np.float64).T, rtol=1e-6)
+    e = np.zeros((4, 16), dtype=np.float32); e[2, 5] = 1.0              # one-hot row picks a column of B
+    D, _ = ob.matmul_nt(e, B[:, :16].copy())
+    assert np.array_equal(D[2], B[:, 5]) and not D[[0, 1, 3]].any()
+
+
 def test_quantize_transposed_is_row_quantize_of_the_transpose():
     rng = np.random.default_rng(8)
     x = torch.from_numpy(rng.standard_normal((32, 24)).astype(np.float32)).to(torch.bfloat16).float().numpy()
