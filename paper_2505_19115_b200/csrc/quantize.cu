@@ -21,7 +21,7 @@ constexpr int kRowTileRows = 128;
 constexpr int kSfChunkPitch = 528;  // 512 + 16: spreads the eight k-tiles over different banks
 
 template <typename T, bool SR, bool SWZ>
-__global__ void __launch_bounds__(kThreads, 3) quantize_row_kernel(const QuantParams p) {
+__global__ void __launch_bounds__(kThreads, (SR && sizeof(T) == 2) ? 4 : 3) quantize_row_kernel(const QuantParams p) {
   __shared__ __align__(16) uint8_t sf_s[SWZ ? 8 * kSfChunkPitch : 16];
   __shared__ float inv_table[128];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
