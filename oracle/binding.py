@@ -48,6 +48,18 @@ def lib():
         L.nvfp4o_quantize_transposed.restype = None
         L.nvfp4o_quantize_transposed.argtypes = q
         L.nvfp4o_dequantize.restype = None
+        L.nvfp4o_e8m0_encode_up.restype = C.c_uint8
+        L.nvfp4o_e8m0_encode_up.argtypes = [C.c_float]
+        L.nvfp4o_e8m0_decode.restype = C.c_float
+        L.nvfp4o_e8m0_decode.argtypes = [C.c_uint8]
+        L.nvfp4o_quantize_mx_rows.restype = None
+        L.nvfp4o_quantize_mx_rows.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_float, C.c_int, C.c_uint64, C.c_uint64,
+                                              C.c_int64, _u8p, _u8p, C.c_int]
+        L.nvfp4o_dequantize_mx.restype = None
+        L.nvfp4o_dequantize_mx.argtypes = [_u8p, _u8p, C.c_float, C.c_int64, C.c_int64, _f32p]
+        L.nvfp4o_gemm_mx.restype = None
+        L.nvfp4o_gemm_mx.argtypes = [_u8p, _u8p, C.c_float, _u8p, _u8p, C.c_float, C.c_int64, C.c_int64, C.c_int64,
+                                     _f32p, _f32p, C.c_int]
         L.nvfp4o_matmul_nt.restype = None
         L.nvfp4o_matmul_nt.argtypes = [_f32p, _f32p, C.c_int64, C.c_int64, C.c_int64, _f32p, _f32p, C.c_int]
         L.nvfp4o_noise_sums.restype = None
@@ -165,6 +177,48 @@ def noise_sums(x, codes, scales, g=1.0):
     lib().nvfp4o_noise_sums(x, np.ascontiguousarray(codes), np.ascontiguousarray(scales), float(np.float32(g)),
                             x.shape[0], x.shape[1], out)
     return float(out[0]), float(out[1])
+
+
+def e8m0_encode_up(v: float) -> int:
+    return int(lib().nvfp4o_e8m0_encode_up(float(np.float32(v))))
+
+
+def e8m0_decode(code: int) -> float:
+    return float(lib().nvfp4o_e8m0_decode(code))
+
+
+def quantize_mx(x, g=1.0, mode=RTN, seed=0, offset=0, transposed=False, first_row=0, nthreads=None):
+    """MXFP4: blocks of 32 along the quantized rows, E8M0 scales.  Returns (codes [Rq, Kq/2], scales [Rq, Kq/32]).
+    transposed: quantize the transpose of x (blocks along x's rows)."""
+    x = _f32(x)
+    if transposed:
+        x = np.ascontiguousarray(x.T)
+    Rq, Kq = x.shape
+    assert Kq % 32 == 0
+    codes = np.zeros((Rq, Kq // 2), dtype=np.uint8)
+    scales = np.zeros((Rq, Kq // 32), dtype=np.uint8)
+    lib().nvfp4o_quantize_mx_rows(x, Rq, Kq, float(np.float32(g)), mode, seed, offset, first_row, codes, scales,
+                                  host_threads() if nthreads is None else nthreads)
+    return codes, scales
+
+
+def dequantize_mx(codes, scales, g=1.0):
+    Rq, half = codes.shape
+    out = np.zeros((Rq, half * 2), dtype=np.float32)
+    lib().nvfp4o_dequantize_mx(np.ascontiguousarray(codes), np.ascontiguousarray(scales), float(np.float32(g)), Rq,
+                               half * 2, out)
+    return out
+
+
+def gemm_mx(a_codes, a_sf, ga, b_codes, b_sf, gb, nthreads=None):
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    N = b_codes.shape[0]
+    D = np.zeros((M, N), dtype=np.float32)
+    T = np.zeros((M, N), dtype=np.float32)
+    lib().nvfp4o_gemm_mx(np.ascontiguousarray(a_codes), np.ascontiguousarray(a_sf), float(np.float32(ga)),
+                         np.ascontiguousarray(b_codes), np.ascontiguousarray(b_sf), float(np.float32(gb)), M, N, K, D, T,
+                         host_threads() if nthreads is None else nthreads)
+    return D, T
 
 
 def matmul_nt(A, B, nthreads=None):

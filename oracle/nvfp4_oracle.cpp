@@ -188,6 +188,95 @@ void nvfp4o_quantize_rows(const float* x, int64_t Rq, int64_t Kq, float g, int m
   });
 }
 
+// ---------------------------------------------------------------------------------------------
+// MXFP4 (Section 3, Table 1): the same E2M1 elements in blocks of 32 with an E8M0 (power of two)
+// scale.  Readings where the paper is silent: the scale is amax * ((1/6)/g) rounded UP to a power
+// of two (so no element exceeds 6 and nothing clips), code 0 flushes the block; the random
+// integers of SR are drawn per group of 16 elements exactly as for NVFP4.
+// ---------------------------------------------------------------------------------------------
+uint8_t nvfp4o_e8m0_encode_up(float v) {
+  if (!(v > 0.0f)) return 0;
+  int e;
+  float m = std::frexp(v, &e);                                 // v = m * 2^e, m in [0.5, 1)
+  int code = ((m == 0.5f) ? e - 1 : e) + 127;                  // smallest power of two >= v
+  return (uint8_t)(code < 0 ? 0 : (code > 254 ? 254 : code));
+}
+
+float nvfp4o_e8m0_decode(uint8_t code) { return std::ldexp(1.0f, (int)code - 127); }
+
+void nvfp4o_quantize_mx_rows(const float* x, int64_t Rq, int64_t Kq, float g, int mode,
+                             uint64_t seed, uint64_t offset, int64_t first_row,
+                             uint8_t* codes, uint8_t* scales, int nthreads) {
+  const int64_t nkb = Kq / 32, n16 = Kq / 16;
+  const float c = (1.0f / 6.0f) / g;
+  parallel_rows(Rq, nthreads, [=](int64_t r0, int64_t r1) {
+    for (int64_t r = r0; r < r1; ++r) {
+      for (int64_t kb = 0; kb < nkb; ++kb) {
+        const float* xb = x + r * Kq + kb * 32;
+        float amax = 0.0f;
+        for (int j = 0; j < 32; ++j) { float a = std::fabs(xb[j]); if (a > amax) amax = a; }
+        uint8_t s_q = nvfp4o_e8m0_encode_up(amax * c);
+        float d = nvfp4o_e8m0_decode(s_q) * g;
+        float inv = (s_q == 0) ? 0.0f : 1.0f / d;
+        uint8_t nib[32];
+        for (int h = 0; h < 2; ++h) {                          // the two groups of 16 of this block
+          uint16_t rnd[16];
+          if (mode == 1) nvfp4o_block_random_u16(seed, offset, (uint64_t)((first_row + r) * n16 + kb * 2 + h), rnd);
+          for (int j = 0; j < 16; ++j) {
+            float xv = xb[16 * h + j];
+            float y = std::fabs(xv) * inv;
+            y = (y < 6.0f) ? y : 6.0f;
+            uint8_t m = (mode == 1) ? nvfp4o_round_sr(y, rnd[j]) : nvfp4o_round_rtn(y);
+            nib[16 * h + j] = (uint8_t)((std::signbit(xv) ? 8 : 0) | m);
+          }
+        }
+        uint8_t* cb = codes + (r * Kq + kb * 32) / 2;
+        for (int j = 0; j < 16; ++j) cb[j] = (uint8_t)(nib[2 * j] | (nib[2 * j + 1] << 4));
+        scales[r * nkb + kb] = s_q;
+      }
+    }
+  });
+}
+
+void nvfp4o_dequantize_mx(const uint8_t* codes, const uint8_t* scales, float g, int64_t Rq, int64_t Kq, float* out) {
+  const int64_t nkb = Kq / 32;
+  for (int64_t r = 0; r < Rq; ++r)
+    for (int64_t k = 0; k < Kq; ++k) {
+      uint8_t byte = codes[(r * Kq + k) / 2];
+      uint8_t nib = (k & 1) ? (byte >> 4) : (byte & 15);
+      out[r * Kq + k] = code_value(nib) * (nvfp4o_e8m0_decode(scales[r * nkb + k / 32]) * g);
+    }
+}
+
+void nvfp4o_gemm_mx(const uint8_t* a_codes, const uint8_t* a_sf, float ga,
+                    const uint8_t* b_codes, const uint8_t* b_sf, float gb,
+                    int64_t M, int64_t N, int64_t K, float* D, float* T, int nthreads) {
+  const double alpha = (double)ga * (double)gb;
+  const int64_t nkb = K / 32;
+  parallel_rows(M, nthreads, [=](int64_t i0, int64_t i1) {
+    for (int64_t i = i0; i < i1; ++i)
+      for (int64_t j = 0; j < N; ++j) {
+        double acc = 0.0, aabs = 0.0;
+        for (int64_t kb = 0; kb < nkb; ++kb) {
+          double inner = 0.0, inner_abs = 0.0;
+          for (int k = 0; k < 32; ++k) {
+            int64_t kk = kb * 32 + k;
+            uint8_t ab = a_codes[(i * K + kk) / 2], bb = b_codes[(j * K + kk) / 2];
+            double av = code_value((kk & 1) ? (ab >> 4) : (ab & 15));
+            double bv = code_value((kk & 1) ? (bb >> 4) : (bb & 15));
+            inner += av * bv;
+            inner_abs += std::fabs(av * bv);
+          }
+          double sc = (double)nvfp4o_e8m0_decode(a_sf[i * nkb + kb]) * (double)nvfp4o_e8m0_decode(b_sf[j * nkb + kb]);
+          acc += sc * inner;
+          aabs += sc * inner_abs;
+        }
+        if (D) D[i * N + j] = (float)(alpha * acc);
+        if (T) T[i * N + j] = (float)(std::fabs(alpha) * aabs);
+      }
+  });
+}
+
 void nvfp4o_quantize_transposed(const float* x, int64_t rows, int64_t cols, float g, int mode,
                                 uint64_t seed, uint64_t offset,
                                 uint8_t* codes, uint8_t* scales, int nthreads) {

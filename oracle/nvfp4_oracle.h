@@ -71,6 +71,21 @@ void nvfp4o_quantize_rows(const float* x, int64_t Rq, int64_t Kq, float g, int m
                           uint64_t seed, uint64_t offset, int64_t first_row,
                           uint8_t* codes, uint8_t* scales, int nthreads);
 
+/* MXFP4 (Section 3, Table 1): E2M1 elements in blocks of 32 along Kq with an E8M0 scale.
+ * e8m0 code c means 2^(c-127); encode_up gives the smallest power of two >= v (0 for v <= 0, which
+ * flushes the block).  Scale = encode_up(amax * ((1/6)/g)); elements as for NVFP4; the random
+ * integers of SR belong to groups of 16 elements, group index (first_row+r)*(Kq/16) + k/16.
+ * codes: Rq*Kq/2 bytes; scales: linear [Rq, Kq/32].  Kq % 32 == 0. */
+uint8_t nvfp4o_e8m0_encode_up(float v);
+float nvfp4o_e8m0_decode(uint8_t code);
+void nvfp4o_quantize_mx_rows(const float* x, int64_t Rq, int64_t Kq, float g, int mode,
+                             uint64_t seed, uint64_t offset, int64_t first_row,
+                             uint8_t* codes, uint8_t* scales, int nthreads);
+void nvfp4o_dequantize_mx(const uint8_t* codes, const uint8_t* scales, float g, int64_t Rq, int64_t Kq, float* out);
+void nvfp4o_gemm_mx(const uint8_t* a_codes, const uint8_t* a_sf, float ga,
+                    const uint8_t* b_codes, const uint8_t* b_sf, float gb,
+                    int64_t M, int64_t N, int64_t K, float* D, float* T, int nthreads);
+
 /* Transposed quantization of x[rows, cols]: by definition nvfp4o_quantize
  * applied to the materialised transpose (Rq = cols, Kq = rows). */
 void nvfp4o_quantize_transposed(const float* x, int64_t rows, int64_t cols, float g, int mode,

@@ -506,3 +506,79 @@ def test_gemm_transposed_operand_detected():
     A, B = ob.dequantize(ac, asf).astype(np.float64), ob.dequantize(bc, bsf).astype(np.float64)
     assert D.shape == (3, 5)
     assert np.allclose(D, A @ B.T, rtol=1e-6)
+
+
+# ---------------------------------------------------------------- MXFP4 (blocks of 32, E8M0 scales)
+def test_e8m0_is_the_power_of_two_ladder_and_encode_rounds_up():
+    import math
+    for code in range(0, 255):
+        assert ob.e8m0_decode(code) == math.ldexp(1.0, code - 127)
+        assert ob.e8m0_encode_up(ob.e8m0_decode(code)) == code               # powers of two map to themselves
+    rng = np.random.default_rng(41)
+    for v in np.concatenate([rng.uniform(1e-30, 1e30, 300), 2.0 ** rng.uniform(-120, 120, 300)]).astype(np.float32):
+        c = ob.e8m0_encode_up(float(v))
+        assert Fraction(ob.e8m0_decode(c)) >= Fraction(float(v))             # never below the value ...
+        assert c == 0 or Fraction(ob.e8m0_decode(c - 1)) < Fraction(float(v))   # ... and the smallest such power
+    assert ob.e8m0_encode_up(0.0) == 0 and ob.e8m0_encode_up(float(np.float32(3e38))) == 254
+
+
+def test_mx_block_quantizer_by_exhaustive_definition():
+    rng = np.random.default_rng(42)
+    x = torch.from_numpy((rng.standard_normal((6, 96)) * rng.choice([1e-3, 1.0, 40.0], (6, 1))).astype(np.float32)) \
+        .to(torch.bfloat16).float().numpy()
+    codes, scales = ob.quantize_mx(x, nthreads=1)
+    assert codes.shape == (6, 48) and scales.shape == (6, 3)
+    for r in range(6):
+        for kb in range(3):
+            blk = x[r, kb * 32:(kb + 1) * 32]
+            amax = Fraction(float(np.max(np.abs(blk))))
+            d = Fraction(ob.e8m0_decode(int(scales[r, kb])))
+            assert d * 6 >= amax * Fraction(1 - 2 ** -20) and d * 3 < amax * Fraction(1 + 2 ** -20)   # amax/d in (3, 6]
+            for j in range(32):
+                byte = codes[r, (kb * 32 + j) // 2]
+                nib = (byte >> 4) if j & 1 else (byte & 15)
+                y = Fraction(float(abs(blk[j]))) / d
+                dist = [abs(y - g) for g in GRID_F]
+                assert dist[nib & 7] == min(dist) and (nib >> 3) == int(np.signbit(blk[j]))
+    # nothing clips: the largest element of every block lands on code 5, 6 or 7 (3 < y <= 6)
+    assert np.all(np.maximum((codes & 7), (codes >> 4) & 7).reshape(6, 3, 16).max(axis=2) >= 5)
+    deq = ob.dequantize_mx(codes, scales)
+    d_all = np.array([[ob.e8m0_decode(int(b)) for b in row] for row in scales]).repeat(32, axis=1)
+    assert np.all(np.abs(deq - x) <= d_all)                  # half of the widest grid step (2) times the scale
+
+
+def test_mx_sr_draws_per_group_of_16_like_nvfp4_and_slices_compose():
+    rng = np.random.default_rng(43)
+    x = torch.from_numpy(rng.standard_normal((9, 64)).astype(np.float32)).to(torch.bfloat16).float().numpy()
+    c, s_ = ob.quantize_mx(x, mode=ob.SR, seed=5, offset=2, nthreads=1)
+    for r in range(9):
+        for k16 in range(4):
+            rnd = ob.block_random_u16(5, 2, r * 4 + k16)
+            inv = np.float32(1.0) / np.float32(ob.e8m0_decode(int(s_[r, k16 // 2])))
+            for j in range(16):
+                v = x[r, k16 * 16 + j]
+                y = min(np.float32(abs(v)) * inv, np.float32(6.0))
+                byte = c[r, (k16 * 16 + j) // 2]
+                nib = (byte >> 4) if j & 1 else (byte & 15)
+                assert nib == (ob.round_sr(float(y), int(rnd[j])) | (8 if np.signbit(v) else 0))
+    c2, s2 = ob.quantize_mx(x[3:7], mode=ob.SR, seed=5, offset=2, first_row=3, nthreads=2)
+    assert np.array_equal(c[3:7], c2) and np.array_equal(s_[3:7], s2)
+    # transposed = row quantization of the materialised transpose
+    y = np.ascontiguousarray(x[:, :32])                                              # [9, 32] -> transpose has Kq = 9: pad rows
+    y = np.concatenate([y, np.zeros((23, 32), dtype=np.float32)])                    # [32, 32]
+    ct, st = ob.quantize_mx(y, mode=ob.SR, seed=5, offset=2, transposed=True)
+    cr, sr_ = ob.quantize_mx(np.ascontiguousarray(y.T), mode=ob.SR, seed=5, offset=2)
+    assert np.array_equal(ct, cr) and np.array_equal(st, sr_)
+
+
+def test_mx_gemm_against_float64_matmul_of_dequantized_operands():
+    rng = np.random.default_rng(44)
+    A = rng.standard_normal((20, 128)).astype(np.float32)
+    B = (rng.standard_normal((12, 128)) * 0.03).astype(np.float32)
+    ac, asf = ob.quantize_mx(A, g=0.5)
+    bc, bsf = ob.quantize_mx(B, g=0.25)
+    D, T = ob.gemm_mx(ac, asf, 0.5, bc, bsf, 0.25, nthreads=2)
+    da = ob.dequantize_mx(ac, asf, 0.5).astype(np.float64)
+    db = ob.dequantize_mx(bc, bsf, 0.25).astype(np.float64)
+    assert np.allclose(D, da @ db.T, rtol=1e-6, atol=1e-9)
+    assert np.allclose(T, np.abs(da) @ np.abs(db).T, rtol=1e-6)
