@@ -245,6 +245,26 @@ NVFP4_API int nvfp4_linear_bwd(const void* dY, const void* W, const void* X, int
                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * MXFP4 (Section 3, Table 1: the format the paper compares NVFP4 with): the same E2M1 elements in
+ * blocks of 32 along Kq with an E8M0 (power-of-two) scale, scale = amax * ((1/6)/g) rounded UP to a
+ * power of two, so that no element exceeds 6.  Codes as for NVFP4; scales one byte per 32 elements,
+ * linear [Rq, Kq/32] or in the same 128-row x 4-block tiles of 512 bytes (a tile then covers 128
+ * values); nvfp4_sf_bytes_mx gives the size.  The random integers of SR belong to groups of 16
+ * elements exactly as for NVFP4 (group index r*(Kq/16) + k/16).  Kq % 32 == 0.
+ * nvfp4_quantize_mx: transposed == 1 (bf16 only) transposes into `workspace` (rows*cols*2 bytes,
+ * 16-byte aligned) and quantizes the rows of the transpose; workspace may be NULL otherwise.
+ * nvfp4_gemm_mx: as nvfp4_gemm on MXFP4 operands (tcgen05 kind::mxf4, scale_vec::2X).
+ */
+NVFP4_API size_t nvfp4_sf_bytes_mx(int64_t Rq, int64_t Kq, int sf_layout);
+NVFP4_API int nvfp4_quantize_mx(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int transposed,
+                      const float* global_scale, const nvfp4_rounding* rounding /* host */,
+                      uint8_t* codes, uint8_t* scales, int sf_layout,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
+NVFP4_API int nvfp4_gemm_mx(const uint8_t* a_codes, const uint8_t* a_sf, const float* a_g,
+                  const uint8_t* b_codes, const uint8_t* b_sf, const float* b_g,
+                  int64_t M, int64_t N, int64_t K, void* d, int d_dtype, int64_t ldd, void* cuda_stream);
+
+/*
  * Quantization-aware fine-tuning phase (Section 5): the forward pass stays in NVFP4
  * (nvfp4_linear_fwd), the backward and update products run in BF16.
  *

@@ -81,6 +81,12 @@ def lib():
     L.nvfp4_linear_bwd_saved.argtypes = [vp, ci, i64, i64, i64, ci, vp, rp, rp, vp, sz, vp, ci, vp, ci, vp, sz, vp]
     L.nvfp4_linear_bwd.restype = ci
     L.nvfp4_linear_bwd.argtypes = [vp, vp, vp, ci, i64, i64, i64, ci, vp, vp, vp, rp, rp, rp, rp, vp, ci, vp, ci, vp, sz, vp]
+    L.nvfp4_sf_bytes_mx.restype = sz
+    L.nvfp4_sf_bytes_mx.argtypes = [i64, i64, ci]
+    L.nvfp4_quantize_mx.restype = ci
+    L.nvfp4_quantize_mx.argtypes = [vp, ci, i64, i64, i64, ci, vp, rp, vp, vp, ci, vp, sz, vp]
+    L.nvfp4_gemm_mx.restype = ci
+    L.nvfp4_gemm_mx.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, i64, vp]
     L.nvfp4_gemm_bf16.restype = ci
     L.nvfp4_gemm_bf16.argtypes = [vp, vp, i64, i64, i64, vp, ci, i64, vp]
     L.nvfp4_transpose_bf16.restype = ci
@@ -337,6 +343,42 @@ def nvfp4_linear_bwd(dY, W, X, gscale_mode=G_AMAX, gdy=None, gw=None, gx=None, r
                                 _ptr(dX), _dtype_code(dX), _ptr(dW), _dtype_code(dW), _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "nvfp4_linear_bwd")
     return dX, dW
+
+
+def nvfp4_sf_bytes_mx(Rq: int, Kq: int, sf_layout: int = SF_SWIZZLED) -> int:
+    return int(lib().nvfp4_sf_bytes_mx(Rq, Kq, sf_layout))
+
+
+def nvfp4_quantize_mx(x, transposed: bool = False, global_scale=None, rounding: Rounding = None,
+                      sf_layout: int = SF_LINEAR, stream=None):
+    """MXFP4 (blocks of 32, E8M0 scales).  Returns (codes [Rq, Kq/2], scales: [Rq, Kq/32] or a flat swizzled buffer)."""
+    assert x.is_cuda and x.dim() == 2 and x.stride(1) == 1
+    rows, cols = x.shape
+    Rq, Kq = (cols, rows) if transposed else (rows, cols)
+    rounding = rounding or Rounding()
+    codes = torch.empty((Rq, Kq // 2), dtype=torch.uint8, device=x.device)
+    if sf_layout == SF_LINEAR:
+        scales = torch.empty((Rq, Kq // 32), dtype=torch.uint8, device=x.device)
+    else:
+        scales = torch.empty(max(nvfp4_sf_bytes_mx(Rq, Kq, sf_layout), 16), dtype=torch.uint8, device=x.device)
+    ws = torch.empty(rows * cols * 2, dtype=torch.uint8, device=x.device) if transposed else None
+    st = lib().nvfp4_quantize_mx(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), int(transposed), _ptr(global_scale),
+                                 C.byref(rounding), _ptr(codes), _ptr(scales), sf_layout, _ptr(ws),
+                                 ws.numel() if ws is not None else 0, _stream(stream))
+    _check(st, "nvfp4_quantize_mx")
+    return codes, scales
+
+
+def nvfp4_gemm_mx(a_codes, a_sf, a_g, b_codes, b_sf, b_g, out_dtype=torch.float32, out=None, stream=None):
+    """D[M,N] = A[M,K] . B[N,K]^T on MXFP4 operands with swizzled E8M0 scales."""
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    N = b_codes.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=a_codes.device)
+    st = lib().nvfp4_gemm_mx(_ptr(a_codes), _ptr(a_sf), _ptr(a_g), _ptr(b_codes), _ptr(b_sf), _ptr(b_g), M, N, K,
+                             _ptr(out), _dtype_code(out), out.stride(0), _stream(stream))
+    _check(st, "nvfp4_gemm_mx")
+    return out
 
 
 def nvfp4_gemm_bf16(A, B, out_dtype=torch.float32, out=None, stream=None):

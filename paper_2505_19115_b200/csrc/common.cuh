@@ -41,6 +41,14 @@ __device__ __forceinline__ uint32_t e4m3_encode(float v) {
   return r & 0xFFu;
 }
 
+// E8M0 (power-of-two) scale of MXFP4: the smallest power of two >= v, as code = exponent + 127
+// (0 for v <= 0 or below 2^-127, 254 at most).
+__device__ __forceinline__ uint32_t e8m0_encode_up(float v) {
+  uint16_t r;
+  asm("cvt.rp.satfinite.ue8m0x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.0f), "f"(v));
+  return (v > 0.0f) ? (r & 0xFFu) : 0u;
+}
+
 // Exact value of an unsigned E4M3 code (0..0x7E).
 __device__ __forceinline__ float e4m3_decode(uint32_t q) {
   return (q < 8u) ? __uint2float_rn(q) * 0x1p-9f : __uint_as_float((q << 20) + (120u << 23));

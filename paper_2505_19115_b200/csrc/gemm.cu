@@ -56,7 +56,8 @@ struct GemmParams {
   int64_t ldd;
   int M, N, K;
   int tiles_m, tiles_n, k_stages;   // k_stages = ceil(K / 256)
-  int k_tiles;                      // ceil(K / 64): 512-byte scale tiles per row tile
+  int k_tiles;                      // 512-byte scale tiles per row tile: ceil(K / 64) (NVFP4), ceil(K / 128) (MXFP4)
+  int k_mmas;                       // instructions along K
   int a_row_tiles, b_row_tiles;     // ceil(M / 128), ceil(N / 128)
   int d_is_bf16;
 };
@@ -287,6 +288,16 @@ __device__ __forceinline__ void tc_mma_nvf4_pair(uint32_t d_tmem, uint64_t adesc
                : "memory");
 }
 
+// MXFP4: blocks of 32 with UE8M0 scales (two scales per row per instruction)
+__device__ __forceinline__ void tc_mma_mxf4_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile("{\n\t.reg .pred p;\n\t"
+               "setp.ne.b32 p, %4, 0;\n\t"
+               "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
+               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+               : "memory");
+}
+
 // bf16 x bf16 -> fp32, 256 x N x 16 per instruction (the backward / update products of the paper's
 // quantization-aware fine-tuning phase, which run in BF16)
 __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
@@ -313,6 +324,12 @@ __device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
 // Instruction descriptor of kind::f16 with bf16 operands (format 1) and an fp32 accumulator (bit 4).
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+// Instruction descriptor of kind::mxf4 (scale_vec::2X): as above with UE8M0 scales (bit 23) and the
+// half of the 32-bit scale column to use (bytes 0-1 or 2-3) at bits 4-5 (B) and 29-30 (A).
+__host__ __device__ constexpr uint32_t instr_desc_mx(int m, int n, int sf_half) {
+  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(m >> 4) << 24) |
+         ((uint32_t)(2 * sf_half) << 4) | ((uint32_t)(2 * sf_half) << 29);
 }
 __host__ __device__ constexpr uint32_t instr_desc(int m, int n) {
   return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (0u << 23) | ((uint32_t)(m >> 4) << 24);
@@ -568,6 +585,7 @@ struct Gemm2Params {
   const float* b_g;
   int M, N, K;
   int tiles_m, tiles_n, k_stages, k_tiles;
+  int k_mmas;                       // instructions along K (64 values each; 16 for bf16 operands)
   int a_row_tiles, b_row_tiles;
   // quantized output (OUT == 2): per-tensor scale of the output, rounding, scales destination
   const float* out_g;
@@ -582,7 +600,10 @@ struct Gemm2Params {
 // round trip through memory.
 // BF16_IN: operands are plain bf16 [rows, K] (K-major) instead of packed codes with scales; the scale
 // producer and the scale movers then have nothing to do and a k-stage is 64 values (128 bytes per row).
-template <int BN, int OUT, bool BF16_IN = false>
+// MX: MXFP4 operands (blocks of 32, E8M0 scales): a 512-byte scale tile then covers 128 values, a
+// stage holds two tiles per 128 rows instead of four, and two consecutive instructions share a
+// scale column, each using one half of it.
+template <int BN, int OUT, bool BF16_IN = false, bool MX = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemm2Threads, 1)
 gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
@@ -667,7 +688,8 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     int s = 0;
     uint32_t ph = 0;
     bool ok = true;
-    constexpr uint32_t kScaleTx = C::kSfaBytes + C::kSfbBytes;     // signalled on this CTA's own barrier
+    constexpr int kSfTiles = MX ? 2 : 4;                           // 512-byte scale tiles per stage and 128 rows
+    constexpr uint32_t kScaleTx = (C::kSfaBytes + C::kSfbBytes) / 4 * kSfTiles;   // signalled on this CTA's own barrier
     for (int tile = pair; !BF16_IN && ok && tile < num_tiles; tile += num_pairs) {
       int tm, tn;
       tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
@@ -681,10 +703,10 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         const uint32_t sf = smem_base + s * C::kStageBytes + C::kABytes + C::kBBytes;
         if (issuer) {
           mbar_arrive_expect_tx(sfl_bar(s), kScaleTx);
-          tma_load_2d(sf, &map_sfa, sfl_bar(s), 0, a_row + ks * 4);
+          tma_load_2d(sf, &map_sfa, sfl_bar(s), 0, a_row + ks * kSfTiles);
 #pragma unroll
           for (int h = 0; h < C::kSfbTiles; ++h)
-            tma_load_2d(sf + C::kSfaBytes + h * 2048, &map_sfb, sfl_bar(s), 0, b_row[h] + ks * 4);
+            tma_load_2d(sf + C::kSfaBytes + h * 2048, &map_sfb, sfl_bar(s), 0, b_row[h] + ks * kSfTiles);
         }
         if (++s == C::kStages) { s = 0; ph ^= 1u; }
       }
@@ -714,13 +736,19 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
           }
           tc_fence_after();
           const uint32_t st = smem_base + s * C::kStageBytes;
-          const int nkt = min(4, p.k_tiles - ks * 4);
+          const int nkt = min(4, p.k_mmas - ks * 4);
           const uint32_t sfa_t = tmem_base + C::kSfaCol + b * C::kSfCols;
           const uint32_t sfb_t = sfa_t + 16 + sfb_off;
           const uint64_t adesc = operand_desc(st), bdesc = operand_desc(st + C::kABytes);
           if (issuer && BF16_IN) {
             for (int j = 0; j < nkt; ++j) tc_mma_bf16_pair(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, (ks | j) ? 1u : 0u);
             tc_commit_pair(empty_bar(s));
+          } else if (issuer && MX) {
+            for (int j = 0; j < nkt; ++j)
+              tc_mma_mxf4_pair(d_tmem, adesc + 2u * j, bdesc + 2u * j, (j & 1) ? instr_desc_mx(256, BN, 1) : instr_desc_mx(256, BN, 0),
+                               sfa_t + 4 * (j >> 1), sfb_t + 4 * C::kSfbTiles * (j >> 1), (ks | j) ? 1u : 0u);
+            tc_commit_pair(empty_bar(s));
+            if constexpr (!C::kSfFollowsStage) tc_commit_pair(sfe_bar(b));
           } else if (issuer) {
             if (nkt == 4) {
 #pragma unroll
@@ -980,12 +1008,12 @@ bool make_codes_map(CUtensorMap* map, const uint8_t* base, int64_t rows, int64_t
 }
 
 // Scale tiles as a 2-D tensor of 32-bit words: one 512-byte tile per row, boxes of four tiles.
-bool make_sf_map(CUtensorMap* map, const uint8_t* base, int64_t n_tiles) {
+bool make_sf_map(CUtensorMap* map, const uint8_t* base, int64_t n_tiles, int box_tiles = 4) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {128, (cuuint64_t)n_tiles};
   const cuuint64_t strides[1] = {512};
-  const cuuint32_t box[2] = {128, 4};
+  const cuuint32_t box[2] = {128, (cuuint32_t)box_tiles};
   const cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<uint8_t*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1057,7 +1085,7 @@ bool make_qout_map(CUtensorMap* map, uint8_t* base, int64_t M, int64_t N) {
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int OUT, bool BF16_IN = false>
+template <int BN, int OUT, bool BF16_IN = false, bool MX = false>
 int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParams& g, cudaStream_t s,
                  const QuantOut& q = QuantOut()) {
   using C = Cfg2<BN>;
@@ -1069,8 +1097,8 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
     map_sfa = map_a;                                                     // never used by the kernel
     map_sfb = map_b;
   } else {
-    if (!make_sf_map(&map_sfa, g.a_sf, (int64_t)g.a_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
-    if (!make_sf_map(&map_sfb, g.b_sf, (int64_t)g.b_row_tiles * g.k_tiles)) return NVFP4_ERR_CUDA;
+    if (!make_sf_map(&map_sfa, g.a_sf, (int64_t)g.a_row_tiles * g.k_tiles, MX ? 2 : 4)) return NVFP4_ERR_CUDA;
+    if (!make_sf_map(&map_sfb, g.b_sf, (int64_t)g.b_row_tiles * g.k_tiles, MX ? 2 : 4)) return NVFP4_ERR_CUDA;
   }
   if constexpr (OUT == 2) {
     if (!make_qout_map(&map_d, q.codes, g.M, g.N)) return NVFP4_ERR_CUDA;
@@ -1082,6 +1110,7 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
   p.tiles_m = (g.M + 255) / 256;
   p.tiles_n = (g.N + BN - 1) / BN;
   p.k_stages = g.k_stages; p.k_tiles = g.k_tiles;
+  p.k_mmas = g.k_mmas;
   p.a_row_tiles = g.a_row_tiles; p.b_row_tiles = g.b_row_tiles;
   p.out_g = q.g; p.out_scales = q.scales; p.out_sr = 0; p.out_swizzled = q.sf_layout == NVFP4_SF_SWIZZLED_128x4;
   p.out_nkb = g.N / 16; p.out_k_tiles = ceil_div(p.out_nkb, 4);
@@ -1089,7 +1118,7 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
   if (q.rounding) p.out_sr = q.rounding->mode == NVFP4_SR;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm2_nvfp4_kernel<BN, OUT, BF16_IN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(gemm2_nvfp4_kernel<BN, OUT, BF16_IN, MX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::kSmemBytes) != cudaSuccess)
       return NVFP4_ERR_CUDA;
     attr_set = true;
@@ -1097,7 +1126,7 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
   const int tiles = p.tiles_m * p.tiles_n;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  gemm2_nvfp4_kernel<BN, OUT, BF16_IN><<<2 * pairs, kGemm2Threads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
+  gemm2_nvfp4_kernel<BN, OUT, BF16_IN, MX><<<2 * pairs, kGemm2Threads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
   return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
@@ -1142,6 +1171,7 @@ extern "C" int nvfp4_gemm(const uint8_t* a_codes, const uint8_t* a_sf, const flo
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
   p.k_stages = (int)ceil_div(K, BK);
   p.k_tiles = (int)ceil_div(K, MMA_K);
+  p.k_mmas = p.k_tiles;
   p.a_row_tiles = (int)ceil_div(M, 128);
   p.b_row_tiles = (int)ceil_div(N, 128);
   p.d_is_bf16 = (d_dtype == NVFP4_BF16);
@@ -1176,6 +1206,7 @@ extern "C" int nvfp4_gemm_quantized(const uint8_t* a_codes, const uint8_t* a_sf,
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
   p.k_stages = (int)ceil_div(K, BK);
   p.k_tiles = (int)ceil_div(K, MMA_K);
+  p.k_mmas = p.k_tiles;
   p.a_row_tiles = (int)ceil_div(M, 128);
   p.b_row_tiles = (int)ceil_div(N, 128);
   p.d_is_bf16 = 0;
@@ -1183,6 +1214,33 @@ extern "C" int nvfp4_gemm_quantized(const uint8_t* a_codes, const uint8_t* a_sf,
   QuantOut q;
   q.g = out_global_scale; q.rounding = rounding; q.codes = out_codes; q.scales = out_scales; q.sf_layout = sf_layout;
   return launch_gemm2<256, 2>(a_codes, b_codes, p, static_cast<cudaStream_t>(cuda_stream), q);
+}
+
+extern "C" int nvfp4_gemm_mx(const uint8_t* a_codes, const uint8_t* a_sf, const float* a_g,
+                             const uint8_t* b_codes, const uint8_t* b_sf, const float* b_g,
+                             int64_t M, int64_t N, int64_t K, void* d, int d_dtype, int64_t ldd, void* cuda_stream) {
+  if (!a_codes || !a_sf || !b_codes || !b_sf || !d) return NVFP4_ERR_NULL;
+  if (d_dtype != NVFP4_BF16 && d_dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if (M <= 0 || N <= 0 || K <= 0 || (K % 32) != 0 || ldd < N) return NVFP4_ERR_SHAPE;
+  if (M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256 || K >= (1ll << 31) - 256) return NVFP4_ERR_SHAPE;
+  const int64_t esz = (d_dtype == NVFP4_BF16) ? 2 : 4;
+  if (!aligned16(a_codes) || !aligned16(a_sf) || !aligned16(b_codes) || !aligned16(b_sf) || !aligned16(d) ||
+      ((ldd * esz) % 16) != 0)
+    return NVFP4_ERR_ALIGN;
+  if (int st = check_arch()) return st;
+  GemmParams p;
+  p.a_sf = a_sf; p.b_sf = b_sf; p.a_g = a_g; p.b_g = b_g; p.d = d; p.ldd = ldd;
+  p.M = (int)M; p.N = (int)N; p.K = (int)K;
+  p.k_stages = (int)ceil_div(K, BK);
+  p.k_tiles = (int)ceil_div(K, 128);                 // one 512-byte scale tile covers four blocks of 32
+  p.k_mmas = (int)ceil_div(K, MMA_K);
+  p.a_row_tiles = (int)ceil_div(M, 128);
+  p.b_row_tiles = (int)ceil_div(N, 128);
+  p.d_is_bf16 = (d_dtype == NVFP4_BF16);
+  p.tiles_m = p.tiles_n = 0;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  return p.d_is_bf16 ? launch_gemm2<256, 1, false, true>(a_codes, b_codes, p, s)
+                     : launch_gemm2<256, 0, false, true>(a_codes, b_codes, p, s);
 }
 
 extern "C" int nvfp4_gemm_bf16(const void* a, const void* b, int64_t M, int64_t N, int64_t K,
@@ -1199,6 +1257,7 @@ extern "C" int nvfp4_gemm_bf16(const void* a, const void* b, int64_t M, int64_t 
   p.M = (int)M; p.N = (int)N; p.K = (int)K;
   p.k_stages = (int)ceil_div(K * 2, BK_BYTES);       // 64 bf16 values per stage
   p.k_tiles = (int)(K / 16);                         // 32-byte steps = one MMA each
+  p.k_mmas = p.k_tiles;
   p.a_row_tiles = (int)ceil_div(M, 128);
   p.b_row_tiles = (int)ceil_div(N, 128);
   p.d_is_bf16 = (d_dtype == NVFP4_BF16);

@@ -20,10 +20,13 @@ namespace {
 constexpr int kRowTileRows = 128;
 constexpr int kSfChunkPitch = 528;  // 512 + 16: spreads the eight k-tiles over different banks
 
-template <typename T, bool SR, bool SWZ>
+// MX = true is the MXFP4 variant (Section 3, Table 1): blocks of 32 with an E8M0 scale rounded up to a
+// power of two.  A lane still encodes 16 values; the two lanes of a block share their amax by a shuffle
+// and the even lane stores the scale.
+template <typename T, bool SR, bool SWZ, bool MX = false>
 __global__ void __launch_bounds__(kThreads, (SR && sizeof(T) == 2) ? 4 : 3) quantize_row_kernel(const QuantParams p) {
   __shared__ __align__(16) uint8_t sf_s[SWZ ? 8 * kSfChunkPitch : 16];
-  __shared__ float inv_table[128];
+  __shared__ float inv_table[MX ? 256 : 128];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t kb = (int64_t)blockIdx.x * 32 + lane;
   const int64_t row0 = (int64_t)blockIdx.y * kRowTileRows;
@@ -32,8 +35,13 @@ __global__ void __launch_bounds__(kThreads, (SR && sizeof(T) == 2) ? 4 : 3) quan
   const float c = __fdiv_rn(__fdiv_rn(1.0f, 6.0f), g);
   const T* x = static_cast<const T*>(p.x);
   const bool aligned32 = ((reinterpret_cast<uintptr_t>(x) | (uintptr_t)(p.ld * (int64_t)sizeof(T))) & 31u) == 0;
+  // scale position of this lane inside the CTA's 128-row x 32-group tile
+  const int sf_chunk = MX ? (lane >> 3) : (lane >> 2);        // k-tile within the CTA tile
+  const int sf_byte = MX ? ((lane >> 1) & 3) : (lane & 3);
+  const bool sf_owner = MX ? ((lane & 1) == 0) : true;
+  constexpr int kTilesPerCta = MX ? 4 : 8;
 
-  build_inv_table(inv_table, g);
+  if constexpr (MX) build_inv_table_mx(inv_table, g); else build_inv_table(inv_table, g);
   if constexpr (SWZ) {
     for (int i = threadIdx.x; i < 8 * kSfChunkPitch / 16; i += kThreads)
       reinterpret_cast<uint4*>(sf_s)[i] = make_uint4(0, 0, 0, 0);
@@ -53,18 +61,27 @@ __global__ void __launch_bounds__(kThreads, (SR && sizeof(T) == 2) ? 4 : 3) quan
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      if (!ok[u]) continue;
       const int rl = warp + 8 * (it + u);
       const int64_t r = row0 + rl;
       float v[16];
-      const float amax = raw[u].unpack(v);
+      float amax = 0.0f;
+      if (ok[u]) amax = raw[u].unpack(v);
+      if constexpr (MX) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));   // Kq % 32 == 0: both lanes valid or neither
+      if (!ok[u]) continue;
       uint32_t lo, hi, sf;
-      encode_block<SR>(v, amax, c, inv_table, p.rng, (uint64_t)(r * p.nkb + kb), lo, hi, sf);
-      *reinterpret_cast<uint2*>(p.codes + (r * p.nkb + kb) * 8) = make_uint2(lo, hi);
-      if constexpr (SWZ) {
-        sf_s[(lane >> 2) * kSfChunkPitch + (rl & 31) * 16 + (rl >> 5) * 4 + (lane & 3)] = (uint8_t)sf;
+      if constexpr (MX) {
+        sf = e8m0_encode_up(__fmul_rn(amax, c));
+        encode_codes<SR>(v, inv_table[sf], p.rng, (uint64_t)(r * p.nkb + kb), lo, hi);
       } else {
-        p.scales[r * p.nkb + kb] = (uint8_t)sf;
+        encode_block<SR>(v, amax, c, inv_table, p.rng, (uint64_t)(r * p.nkb + kb), lo, hi, sf);
+      }
+      *reinterpret_cast<uint2*>(p.codes + (r * p.nkb + kb) * 8) = make_uint2(lo, hi);
+      if (sf_owner) {
+        if constexpr (SWZ) {
+          sf_s[sf_chunk * kSfChunkPitch + (rl & 31) * 16 + (rl >> 5) * 4 + sf_byte] = (uint8_t)sf;
+        } else {
+          p.scales[r * p.nsb + (MX ? (kb >> 1) : kb)] = (uint8_t)sf;
+        }
       }
     }
   }
@@ -72,8 +89,8 @@ __global__ void __launch_bounds__(kThreads, (SR && sizeof(T) == 2) ? 4 : 3) quan
   if constexpr (SWZ) {
     __syncthreads();
     const int q = threadIdx.x >> 5, i = threadIdx.x & 31;
-    const int64_t kt = (int64_t)blockIdx.x * 8 + q;
-    if (kt < p.k_tiles) {
+    const int64_t kt = (int64_t)blockIdx.x * kTilesPerCta + q;
+    if (q < kTilesPerCta && kt < p.k_tiles) {
       const uint4 val = *reinterpret_cast<const uint4*>(sf_s + q * kSfChunkPitch + i * 16);
       *reinterpret_cast<uint4*>(p.scales + ((int64_t)blockIdx.y * p.k_tiles + kt) * 512 + i * 16) = val;
     }
@@ -359,7 +376,7 @@ extern "C" int nvfp4_quantize(const void* x, int dtype, int64_t rows, int64_t co
   p.x = x; p.rows = rows; p.cols = cols; p.ld = ld; p.gptr = global_scale;
   philox_stream_init(&p.rng, rounding->seed, rounding->offset);
   p.codes = codes; p.scales = scales;
-  p.nkb = Kq / 16; p.k_tiles = ceil_div(p.nkb, 4);
+  p.nkb = Kq / 16; p.nsb = p.nkb; p.k_tiles = ceil_div(p.nsb, 4);
   if (ceil_div(rows, 128) > 65535) return NVFP4_ERR_SHAPE;  // grid.y limit
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   if (transposed && tile_quantizer_eligible(dtype, rows, cols, false))
@@ -368,6 +385,67 @@ extern "C" int nvfp4_quantize(const void* x, int dtype, int64_t rows, int64_t co
   const bool sr = rounding->mode == NVFP4_SR, swz = sf_layout == NVFP4_SF_SWIZZLED_128x4;
   cudaError_t e = (dtype == NVFP4_BF16) ? dispatch<__nv_bfloat16>(p, transposed != 0, sr, swz, s)
                                         : dispatch<float>(p, transposed != 0, sr, swz, s);
+  return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+
+namespace nvfp4 {
+namespace {
+template <typename T>
+cudaError_t dispatch_row_mx(const QuantParams& p, bool sr, bool swz, cudaStream_t s) {
+  dim3 grid((unsigned)ceil_div(p.nkb, 32), (unsigned)ceil_div(p.rows, kRowTileRows));
+  if (sr) {
+    if (swz) quantize_row_kernel<T, true, true, true><<<grid, kThreads, 0, s>>>(p);
+    else quantize_row_kernel<T, true, false, true><<<grid, kThreads, 0, s>>>(p);
+  } else {
+    if (swz) quantize_row_kernel<T, false, true, true><<<grid, kThreads, 0, s>>>(p);
+    else quantize_row_kernel<T, false, false, true><<<grid, kThreads, 0, s>>>(p);
+  }
+  return cudaGetLastError();
+}
+}  // namespace
+}  // namespace nvfp4
+
+extern "C" size_t nvfp4_sf_bytes_mx(int64_t Rq, int64_t Kq, int sf_layout) {
+  if (Rq <= 0 || Kq <= 0 || (Kq % 32) != 0) return 0;
+  if (sf_layout == NVFP4_SF_LINEAR) return (size_t)(Rq * (Kq / 32));
+  if (sf_layout == NVFP4_SF_SWIZZLED_128x4) return (size_t)(ceil_div(Rq, 128) * ceil_div(Kq, 128) * 512);
+  return 0;
+}
+
+extern "C" int nvfp4_quantize_mx(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, int transposed,
+                                 const float* global_scale, const nvfp4_rounding* rounding,
+                                 uint8_t* codes, uint8_t* scales, int sf_layout,
+                                 void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!x || !rounding || !codes || !scales) return NVFP4_ERR_NULL;
+  if (dtype != NVFP4_BF16 && dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if (transposed != 0 && transposed != 1) return NVFP4_ERR_ENUM;
+  if (transposed && dtype != NVFP4_BF16) return NVFP4_ERR_ENUM;        // the transposed path goes through the bf16 transpose
+  if ((rounding->mode != NVFP4_RTN && rounding->mode != NVFP4_SR) || rounding->reserved != 0) return NVFP4_ERR_ENUM;
+  if (sf_layout != NVFP4_SF_LINEAR && sf_layout != NVFP4_SF_SWIZZLED_128x4) return NVFP4_ERR_ENUM;
+  if (rows <= 0 || cols <= 0 || ld < cols || cols % 8 != 0) return NVFP4_ERR_SHAPE;
+  const int64_t Rq = transposed ? cols : rows, Kq = transposed ? rows : cols;
+  if (Kq % 32 != 0 || rows >= (int64_t)1 << 31 || cols >= (int64_t)1 << 31) return NVFP4_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(codes) || !aligned16(scales) || (ld % 8) != 0) return NVFP4_ERR_ALIGN;
+  if (ceil_div(Rq, 128) > 65535) return NVFP4_ERR_SHAPE;
+  if (int st = check_arch()) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const void* src = x;
+  int64_t src_ld = ld;
+  if (transposed) {
+    // Q(x^T) is by definition the row quantization of the materialised transpose
+    if (!workspace || workspace_bytes < (size_t)rows * cols * 2 || (reinterpret_cast<uintptr_t>(workspace) & 15u))
+      return NVFP4_ERR_WORKSPACE;
+    if (int st = nvfp4_transpose_bf16(x, rows, cols, ld, workspace, cuda_stream)) return st;
+    src = workspace;
+    src_ld = rows;
+  }
+  QuantParams p;
+  p.x = src; p.rows = Rq; p.cols = Kq; p.ld = src_ld; p.gptr = global_scale;
+  philox_stream_init(&p.rng, rounding->seed, rounding->offset);
+  p.codes = codes; p.scales = scales;
+  p.nkb = Kq / 16; p.nsb = Kq / 32; p.k_tiles = ceil_div(p.nsb, 4);
+  const bool sr = rounding->mode == NVFP4_SR, swz = sf_layout == NVFP4_SF_SWIZZLED_128x4;
+  cudaError_t e = (dtype == NVFP4_BF16) ? dispatch_row_mx<__nv_bfloat16>(p, sr, swz, s) : dispatch_row_mx<float>(p, sr, swz, s);
   return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 

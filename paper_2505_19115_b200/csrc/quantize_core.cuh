@@ -17,8 +17,9 @@ struct QuantParams {
   PhiloxStream rng;
   uint8_t* codes;
   uint8_t* scales;
-  int64_t nkb;      // blocks per quantized row (Kq / 16)
-  int64_t k_tiles;  // ceil(nkb / 4)
+  int64_t nkb;      // groups of 16 per quantized row (Kq / 16): NVFP4 blocks, and the unit of the random draws
+  int64_t k_tiles;  // scale tiles per quantized row: ceil(scale blocks / 4)
+  int64_t nsb;      // scale blocks per quantized row: Kq / 16 (NVFP4) or Kq / 32 (MXFP4)
 };
 
 // Reciprocal of every block scale a tensor can have: entry q = 1 / (decode(q) * g), one IEEE
@@ -28,15 +29,31 @@ __device__ __forceinline__ void build_inv_table(float* inv_table, float g) {
     inv_table[q] = (q == 0) ? 0.0f : __fdiv_rn(1.0f, __fmul_rn(e4m3_decode((uint32_t)q), g));
 }
 
-// 16 values (signed, already widened to fp32) and their amax -> 8 bytes of codes (lo, hi words)
-// and one scale byte.  c = (1/6)/g.  `blk` is the block's linear index (Philox counter).
+// MXFP4: the same table over the 255 E8M0 codes, entry q = 1 / (2^(q-127) * g), 0 for code 0.
+__device__ __forceinline__ void build_inv_table_mx(float* inv_table, float g) {
+  for (int q = threadIdx.x; q < 256; q += blockDim.x)
+    inv_table[q] = (q == 0 || q == 255) ? 0.0f : __fdiv_rn(1.0f, __fmul_rn(__uint_as_float((uint32_t)q << 23), g));
+}
+
+// 16 values (signed, already widened to fp32) scaled by inv -> 8 bytes of codes (lo, hi words).
+// `blk` is the linear index of this group of 16 (Philox counter).
+template <bool SR>
+__device__ __forceinline__ void encode_codes(const float (&v)[16], float inv, const PhiloxStream& rng, uint64_t blk,
+                                             uint32_t& lo, uint32_t& hi);
+
+// 16 values and their amax -> codes and one E4M3 scale byte.  c = (1/6)/g.
 template <bool SR>
 __device__ __forceinline__ void encode_block(const float (&v)[16], float amax, float c, const float* inv_table,
                                              const PhiloxStream& rng, uint64_t blk,
                                              uint32_t& lo, uint32_t& hi, uint32_t& sf) {
   const uint32_t q = e4m3_encode(__fmul_rn(amax, c));
-  const float inv = inv_table[q];
   sf = q;
+  encode_codes<SR>(v, inv_table[q], rng, blk, lo, hi);
+}
+
+template <bool SR>
+__device__ __forceinline__ void encode_codes(const float (&v)[16], float inv, const PhiloxStream& rng, uint64_t blk,
+                                             uint32_t& lo, uint32_t& hi) {
   float y[16];
 #pragma unroll
   for (int j = 0; j < 16; ++j) y[j] = __fmul_rn(v[j], inv);     // the sign rides along; the conversions clamp at 6
