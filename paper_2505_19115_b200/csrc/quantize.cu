@@ -427,14 +427,14 @@ extern "C" int nvfp4_quantize_mx(const void* x, int dtype, int64_t rows, int64_t
   if (Kq % 32 != 0 || rows >= (int64_t)1 << 31 || cols >= (int64_t)1 << 31) return NVFP4_ERR_SHAPE;
   if (!aligned16(x) || !aligned16(codes) || !aligned16(scales) || (ld % 8) != 0) return NVFP4_ERR_ALIGN;
   if (ceil_div(Rq, 128) > 65535) return NVFP4_ERR_SHAPE;
+  if (transposed && (!workspace || workspace_bytes < (size_t)rows * cols * 2 || (reinterpret_cast<uintptr_t>(workspace) & 15u)))
+    return NVFP4_ERR_WORKSPACE;
   if (int st = check_arch()) return st;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const void* src = x;
   int64_t src_ld = ld;
   if (transposed) {
     // Q(x^T) is by definition the row quantization of the materialised transpose
-    if (!workspace || workspace_bytes < (size_t)rows * cols * 2 || (reinterpret_cast<uintptr_t>(workspace) & 15u))
-      return NVFP4_ERR_WORKSPACE;
     if (int st = nvfp4_transpose_bf16(x, rows, cols, ld, workspace, cuda_stream)) return st;
     src = workspace;
     src_ld = rows;

@@ -88,3 +88,48 @@ def test_gemm_and_linear_argument_errors_are_host_side():
     assert lin(L.nvfp4_linear_fwd, K=528) == 2
     assert lin(L.nvfp4_linear_bwd_dx, N=528) == 2
     assert lin(L.nvfp4_linear_bwd_dw, M=272) == 2
+
+
+def test_newer_entry_points_reject_bad_arguments_on_the_host():
+    L = nb.lib()
+    r = nb.Rounding()
+    rb = C.byref(r)
+    buf = C.c_void_p(0x1000)
+    # both orientations from one read
+    d = lambda **kw: L.nvfp4_quantize_dual(kw.get("x", buf), kw.get("dtype", 0), kw.get("rows", 32), kw.get("cols", 32),
+                                           kw.get("ld", 32), None, kw.get("rr", rb), buf, buf, rb, kw.get("ct", buf), buf,
+                                           kw.get("sf", 0), None)
+    assert d(x=None) == 1 and d(ct=None) == 1 and d(rr=None) == 1
+    assert d(rows=24) == 2 and d(cols=24, ld=24) == 2 and d(ld=16) == 2
+    assert d(dtype=2) == 4 and d(sf=3) == 4
+    assert d(x=C.c_void_p(0x1004)) == 3
+    # fused layer calls: sizes and workspace
+    assert nb.nvfp4_linear_saved_bytes(256, 512, 512) % 256 == 0 and nb.nvfp4_linear_saved_bytes(256, 512, 500) == 0
+    for which in (0, 1, 2):
+        assert nb.nvfp4_linear_fused_workspace_bytes(256, 512, 512, which) > 0
+    assert nb.nvfp4_linear_fused_workspace_bytes(256, 512, 512, 3) == 0
+    fs = lambda **kw: L.nvfp4_linear_fwd_save(kw.get("X", buf), buf, 0, kw.get("M", 256), 512, 512, kw.get("gm", 0), None, None,
+                                              rb, rb, rb, rb, buf, 1, kw.get("sv", buf), kw.get("svb", 1 << 30), buf, 1 << 30, None)
+    assert fs(X=None) == 1 and fs(M=250) == 2 and fs(gm=5) == 4 and fs(sv=None) == 5 and fs(svb=64) == 5 and fs(gm=2) == 1
+    bs = lambda **kw: L.nvfp4_linear_bwd_saved(kw.get("dY", buf), 0, 256, kw.get("N", 512), 512, 0, None, rb, rb, buf, 1 << 30,
+                                               buf, 1, buf, kw.get("dwt", 1), kw.get("ws", buf), 1 << 30, None)
+    assert bs(dY=None) == 1 and bs(N=500) == 2 and bs(dwt=7) == 4 and bs(ws=None) == 5
+    # quantized epilogue, bf16 and MXFP4 products, noise monitor, transpose
+    gq = lambda **kw: L.nvfp4_gemm_quantized(kw.get("a", buf), buf, None, buf, buf, None, 128, kw.get("N", 128), 256, None,
+                                             kw.get("r", rb), buf, buf, kw.get("sf", 0), None)
+    assert gq(a=None) == 1 and gq(r=None) == 1 and gq(N=144) == 2 and gq(sf=9) == 4
+    gb = lambda **kw: L.nvfp4_gemm_bf16(kw.get("a", buf), buf, 128, 128, kw.get("K", 64), buf, kw.get("dt", 1), kw.get("ldd", 128), None)
+    assert gb(a=None) == 1 and gb(K=24) == 2 and gb(dt=5) == 4 and gb(ldd=130) == 3
+    gm = lambda **kw: L.nvfp4_gemm_mx(kw.get("a", buf), buf, None, buf, buf, None, 128, 128, kw.get("K", 256), buf, 1, 128, None)
+    assert gm(a=None) == 1 and gm(K=48) == 2
+    qm = lambda **kw: L.nvfp4_quantize_mx(kw.get("x", buf), kw.get("dtype", 0), 32, kw.get("cols", 64), 64, kw.get("tr", 0), None, rb,
+                                          buf, buf, 0, kw.get("ws", None), 0, None)
+    assert qm(x=None) == 1 and qm(cols=48) == 2 and qm(tr=1, dtype=1) == 4 and qm(tr=1) == 5
+    assert nb.nvfp4_sf_bytes_mx(128, 128, nb.SF_SWIZZLED) == 512 and nb.nvfp4_sf_bytes_mx(3, 64, nb.SF_LINEAR) == 6
+    assert nb.nvfp4_sf_bytes_mx(3, 48, nb.SF_LINEAR) == 0
+    nz = lambda **kw: L.nvfp4_quantization_noise(kw.get("x", buf), 0, 32, kw.get("cols", 32), 32, 0, None, buf, buf, 0,
+                                                 kw.get("sums", buf), None)
+    assert nz(x=None) == 1 and nz(sums=None) == 1 and nz(cols=24) == 2 and nz(sums=C.c_void_p(0x1004)) == 3
+    tr = lambda **kw: L.nvfp4_transpose_bf16(kw.get("x", buf), kw.get("rows", 64), 64, 64, buf, None)
+    assert tr(x=None) == 1 and tr(rows=60) == 2
+    assert L.nvfp4_linear_bwd_bf16_workspace_bytes(256, 512, 512) > 0 and L.nvfp4_linear_bwd_bf16_workspace_bytes(0, 512, 512) == 0
