@@ -24,7 +24,7 @@ constexpr int kSfChunkPitch = 528;  // 512 + 16: spreads the eight k-tiles over 
 // power of two.  A lane still encodes 16 values; the two lanes of a block share their amax by a shuffle
 // and the even lane stores the scale.
 template <typename T, bool SR, bool SWZ, bool MX = false>
-__global__ void __launch_bounds__(kThreads, (SR && sizeof(T) == 2) ? 4 : 3) quantize_row_kernel(const QuantParams p) {
+__global__ void __launch_bounds__(kThreads, 3) quantize_row_kernel(const QuantParams p) {
   __shared__ __align__(16) uint8_t sf_s[SWZ ? 8 * kSfChunkPitch : 16];
   __shared__ float inv_table[MX ? 256 : 128];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
