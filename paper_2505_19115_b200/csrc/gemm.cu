@@ -156,6 +156,14 @@ __device__ __forceinline__ bool elect_one() {
   asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
   return pred != 0;
 }
+// Whole-warp wait of the scale movers, relaxed polls by every lane: these warps issue tcgen05.st, and
+// next to such operations an acquiring poll costs ~180 cycles even when the phase is complete (see
+// mbar_wait_issuer), which with two waits per stage made the movers the slowest role.  What they read
+// afterwards is shared memory written by the bulk copies that completed the phase: the loads follow the
+// poll in program order behind a branch on its result, and shared memory has no cache to go stale.
+__device__ __forceinline__ bool mbar_wait_warp_relaxed(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
+  return mbar_wait_issuer(bar, parity, abort_flag, site);
+}
 // Whole-warp wait: lane 0 polls, then every lane observes the completed phase once itself.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
   bool ok = true;
@@ -573,7 +581,7 @@ struct Cfg2 {
   static constexpr int kSfBufs = kSfBufsFit > kStages ? kStages : kSfBufsFit;
   // with as many scale buffers as stages, buffer b is stage s and needs no barrier of its own
   static constexpr bool kSfFollowsStage = (kSfBufs == kStages);
-  static constexpr int kNumBarriers = 3 * kStages + 2 * kSfBufs + 2 * kAccStages;
+  static constexpr int kNumBarriers = 4 * kStages + 2 * kSfBufs + 2 * kAccStages;
   static_assert(kStageBytes % 1024 == 0, "stage must keep the 1024-byte swizzle alignment");
   static_assert(kSfBufs >= 2, "need at least two scale buffers in tensor memory");
   static_assert(kSmemBytes <= 232448, "shared memory overflow");
@@ -620,6 +628,8 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   // full: operands of both CTAs landed (leader's copy is the one waited on)
   // sfl:  this CTA's scale tiles landed        empty: the stage's MMAs are done (both CTAs)
   // sfr:  scale buffer written in both CTAs (leader's copy)   sfe: scale buffer free again (both CTAs)
+  // sfx:  this CTA's scale tiles of the stage have been read out of shared memory: the slot is refilled then,
+  //       a ring round before the stage's operands, so that scales are in tensor memory before operands land
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto sfl_bar = [&](int s) { return bar_base + 8u * (C::kStages + s); };
   auto empty_bar = [&](int s) { return bar_base + 8u * (2 * C::kStages + s); };
@@ -627,6 +637,7 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   auto sfe_bar = [&](int b) { return bar_base + 8u * (3 * C::kStages + C::kSfBufs + b); };
   auto tfull_bar = [&](int a) { return bar_base + 8u * (3 * C::kStages + 2 * C::kSfBufs + a); };
   auto tempty_bar = [&](int a) { return bar_base + 8u * (3 * C::kStages + 2 * C::kSfBufs + C::kAccStages + a); };
+  auto sfx_bar = [&](int s) { return bar_base + 8u * (3 * C::kStages + 2 * C::kSfBufs + 2 * C::kAccStages + s); };
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(bar_gen + 8 * C::kNumBarriers);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   float* inv_table = reinterpret_cast<float*>(bar_gen + 512);   // OUT == 2 only: 1 / (decode(q) * out_g) per scale code
@@ -638,7 +649,7 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   const int num_tiles = p.tiles_m * p.tiles_n;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(sfl_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int s = 0; s < C::kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(sfl_bar(s), 1); mbar_init(empty_bar(s), 1); mbar_init(sfx_bar(s), 4); }
     for (int b = 0; b < C::kSfBufs; ++b) { mbar_init(sfr_bar(b), 8); mbar_init(sfe_bar(b), 1); }
     for (int a = 0; a < C::kAccStages; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), 8); }
     *abort_flag = 0u;
@@ -699,7 +710,7 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
       for (int h = 0; h < C::kSfbTiles; ++h)                       // rows past N are never stored
         b_row[h] = min((tn * BN) / 128 + h, p.b_row_tiles - 1) * p.k_tiles;
       for (int ks = 0; ks < p.k_stages; ++ks) {
-        if (!(ok = mbar_wait_relaxed(empty_bar(s), ph ^ 1u, abort_flag, 0x18))) break;
+        if (!(ok = mbar_wait_relaxed(sfx_bar(s), ph ^ 1u, abort_flag, 0x18))) break;
         const uint32_t sf = smem_base + s * C::kStageBytes + C::kABytes + C::kBBytes;
         if (issuer) {
           mbar_arrive_expect_tx(sfl_bar(s), kScaleTx);
@@ -783,9 +794,11 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     bool ok = true;
     for (int tile = pair; !BF16_IN && ok && tile < num_tiles; tile += num_pairs) {
       for (int ks = 0; ks < p.k_stages; ++ks) {
-        if (!(ok = mbar_wait_warp(sfl_bar(s), ph, abort_flag, 0x16))) break;
-        if constexpr (!C::kSfFollowsStage) {        // otherwise buffer b == stage s, free once sfl_bar(s) could be armed
-          if (!(ok = mbar_wait_warp(sfe_bar(b), bph ^ 1u, abort_flag, 0x17))) break;
+        if (!(ok = mbar_wait_warp_relaxed(sfl_bar(s), ph, abort_flag, 0x16))) break;
+        if constexpr (!C::kSfFollowsStage) {
+          if (!(ok = mbar_wait_warp_relaxed(sfe_bar(b), bph ^ 1u, abort_flag, 0x17))) break;
+        } else {                                    // buffer b == stage s: free once that stage's previous MMAs are done
+          if (!(ok = mbar_wait_warp_relaxed(empty_bar(s), ph ^ 1u, abort_flag, 0x17))) break;
         }
         tc_fence_after();
         const uint8_t* sf = smem_gen + s * C::kStageBytes + C::kABytes + C::kBBytes + lane * 16;
@@ -810,6 +823,8 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
           }
           tmem_st16(t_sf + 16 + 16 * c, r);
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(sfx_bar(s));     // the tiles are in registers: the slot may be refilled
         tmem_st_wait();
         tc_fence_before();
         __syncwarp();
