@@ -150,3 +150,36 @@ def test_quantized_epilogue_equals_quantizing_the_fp32_product(shape, mode, sf_l
                                   dtype=np.float64).reshape(M, N // 16), 16, axis=1) * g * 2.0
         slack = (1.0 if mode == nb.RTN else 2.0) * step + TOL * T      # also covers the clip of a block's maximum at 6
         assert np.all(np.abs(deq - ref) <= slack)
+
+
+# ---------------------------------------------------------------- the two kernel designs against each other
+@pytest.mark.parametrize("shape", [(4096, 4096, 4096), (2048, 5120, 11008), (5000, 3000, 2080)])
+def test_pair_and_single_cta_kernels_agree_on_large_shapes(shape):
+    # Both kernels add the 64-value products of a row in the same order, so their fp32 results are the
+    # same numbers; a scale tile or a stage consumed one step early or late by either of them would show.
+    M, N, K = shape
+    A = synth.normal((M, K), 1.0, 7, device="cuda")
+    B = synth.normal((N, K), 0.02, 8, device="cuda")
+    ga, gb = nb.nvfp4_tensor_amax_scale(A), nb.nvfp4_tensor_amax_scale(B)
+    ac, asf = nb.nvfp4_quantize(A, global_scale=ga, sf_layout=nb.SF_SWIZZLED)
+    bc, bsf = nb.nvfp4_quantize(B, global_scale=gb, sf_layout=nb.SF_SWIZZLED)
+    outs = {}
+    try:
+        for tile in (256, 2256, 2192):
+            nb.nvfp4_gemm_set_tile_n(tile)
+            for rep in range(3):                          # repeated launches: the result may not depend on timing
+                D = nb.nvfp4_gemm(ac, asf, ga, bc, bsf, gb)
+                if tile in outs:
+                    assert torch.equal(outs[tile], D)
+                outs[tile] = D
+    finally:
+        nb.nvfp4_gemm_set_tile_n(0)
+    assert nb.nvfp4_device_error_word() == 0
+    assert torch.equal(outs[256], outs[2256]) and torch.equal(outs[256], outs[2192])
+    # and a sample of the outputs against the oracle
+    rng = np.random.default_rng(5)
+    ii, jj = rng.integers(0, M, 512), rng.integers(0, N, 512)
+    oa = ob.quantize(A.float().cpu().numpy(), g=float(ga.item()))
+    obq = ob.quantize(B.float().cpu().numpy(), g=float(gb.item()))
+    ref, T = ob.gemm_sampled(oa[0], oa[1], float(ga.item()), obq[0], obq[1], float(gb.item()), ii, jj)
+    assert np.all(np.abs(outs[2256].cpu().numpy()[ii, jj] - ref) <= TOL * T)
