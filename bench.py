@@ -223,7 +223,7 @@ def main():
         for l in layers:
             layer_fwd_bwd(l)
 
-    launches_per_step = len(layers) * (3 * 2 + 3 + 3)     # 3 x (amax + finalize), 3 dual quantizers, 3 GEMMs per layer
+    launches_per_step = len(layers) * (3 + 3 + 3)         # 3 amax sweeps, 3 dual quantizers, 3 GEMMs per layer
     flops_per_step = block_flops(cfg)
 
     def barrier():

@@ -24,6 +24,10 @@ int tile_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, const f
                   const nvfp4_rounding* rr, uint8_t* codes_r, uint8_t* scales_r, int sf_layout, cudaStream_t s);
 int tile_error_word(unsigned int* out);
 
+// Per-tensor scale g = amax/2688 in one launch (quantize.cu); scratch_zeroed: two zeroed 32-bit device words.
+int tensor_amax_scale_ws(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* g_out,
+                         unsigned int* scratch_zeroed, void* cuda_stream);
+
 // ---------------------------------------------------------------------------------------------
 // Scale-factor layout (128 rows x 4 blocks per 512-byte tile, k-tiles contiguous per row tile)
 // ---------------------------------------------------------------------------------------------

@@ -34,16 +34,17 @@ SavedLayout saved_layout(int64_t M, int64_t N, int64_t K) {
   return l;
 }
 
-struct FwdLayout { Operand x, w; size_t total; };
+struct FwdLayout { Operand x, w; size_t scratch, total; };
 FwdLayout fwd_layout(int64_t M, int64_t N, int64_t K) {
   FwdLayout l; size_t off = 0;
   place(off, M, K, &l.x);
   place(off, N, K, &l.w);
+  l.scratch = off; off = align256(off + 64);          // zeroed words of the one-launch amax passes
   l.total = off;
   return l;
 }
 
-struct BwdLayout { Operand dy, dyt, wt, xt; size_t gdy, gw, gx, total; };
+struct BwdLayout { Operand dy, dyt, wt, xt; size_t gdy, gw, gx, scratch, total; };
 BwdLayout bwd_layout(int64_t M, int64_t N, int64_t K, bool with_saved) {
   BwdLayout l; size_t off = 0;
   place(off, M, N, &l.dy);                 // Q(dY): [M, N]
@@ -53,6 +54,7 @@ BwdLayout bwd_layout(int64_t M, int64_t N, int64_t K, bool with_saved) {
   l.gdy = off; off = align256(off + sizeof(float));
   l.gw = off; off = align256(off + sizeof(float));
   l.gx = off; off = align256(off + sizeof(float));
+  l.scratch = off; off = align256(off + 64);
   l.total = off;
   return l;
 }
@@ -68,18 +70,24 @@ bool buffer_ok(const void* p, size_t have, size_t need) {
   return p && have >= need && (reinterpret_cast<uintptr_t>(p) & 255u) == 0;
 }
 
-// Per-tensor scale of one operand according to gscale_mode: NULL, computed into `slot`, or given.
+// Per-tensor scale of one operand according to gscale_mode: NULL, computed into `slot` (one launch, with two
+// zeroed scratch words), or given.
 int resolve_g(int gscale_mode, const void* x, int dtype, int64_t rows, int64_t cols, const float* given, float* slot,
-              void* stream, const float** out) {
+              unsigned int* scratch, void* stream, const float** out) {
   *out = nullptr;
   if (gscale_mode == NVFP4_G_AMAX) {
-    if (int st = nvfp4_tensor_amax_scale(x, dtype, rows, cols, cols, slot, stream)) return st;
+    if (int st = tensor_amax_scale_ws(x, dtype, rows, cols, cols, slot, scratch, stream)) return st;
     *out = slot;
   } else if (gscale_mode == NVFP4_G_GIVEN) {
     if (!given) return NVFP4_ERR_NULL;
     *out = given;
   }
   return NVFP4_OK;
+}
+
+int zero_scratch(int gscale_mode, void* scratch, void* stream) {
+  if (gscale_mode != NVFP4_G_AMAX) return NVFP4_OK;
+  return cudaMemsetAsync(scratch, 0, 64, static_cast<cudaStream_t>(stream)) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
 }  // namespace
@@ -119,17 +127,21 @@ extern "C" int nvfp4_linear_fwd_save(const void* X, const void* W, int dtype, in
   float* sgx = reinterpret_cast<float*>(sv + sl.gx);
   float* sgw = reinterpret_cast<float*>(sv + sl.gw);
   const float *g_x, *g_w;
-  if (int st = resolve_g(gscale_mode, X, dtype, M, K, gx, sgx, cuda_stream, &g_x)) return st;
-  if (int st = resolve_g(gscale_mode, W, dtype, N, K, gw, sgw, cuda_stream, &g_w)) return st;
+  unsigned int* scratch = reinterpret_cast<unsigned int*>(ws + fl.scratch);
+  if (int st = zero_scratch(gscale_mode, scratch, cuda_stream)) return st;
   if (gscale_mode == NVFP4_G_GIVEN) {       // the backward pass reads the scales from `saved`
+    if (!gx || !gw) return NVFP4_ERR_NULL;
     if (cudaMemcpyAsync(sgx, gx, sizeof(float), cudaMemcpyDeviceToDevice, s) != cudaSuccess) return NVFP4_ERR_CUDA;
     if (cudaMemcpyAsync(sgw, gw, sizeof(float), cudaMemcpyDeviceToDevice, s) != cudaSuccess) return NVFP4_ERR_CUDA;
   }
-  if (int st = nvfp4_quantize_dual(X, dtype, M, K, K, g_x, rx, ws + fl.x.codes, ws + fl.x.sf, rxt, sv + sl.xt.codes,
-                                   sv + sl.xt.sf, NVFP4_SF_SWIZZLED_128x4, cuda_stream))
-    return st;
+  // W first: amax(W) leaves the (smaller) weight tensor in L2 for the quantizer that follows it
+  if (int st = resolve_g(gscale_mode, W, dtype, N, K, gw, sgw, scratch, cuda_stream, &g_w)) return st;
   if (int st = nvfp4_quantize_dual(W, dtype, N, K, K, g_w, rw, ws + fl.w.codes, ws + fl.w.sf, rwt, sv + sl.wt.codes,
                                    sv + sl.wt.sf, NVFP4_SF_SWIZZLED_128x4, cuda_stream))
+    return st;
+  if (int st = resolve_g(gscale_mode, X, dtype, M, K, gx, sgx, scratch + 2, cuda_stream, &g_x)) return st;
+  if (int st = nvfp4_quantize_dual(X, dtype, M, K, K, g_x, rx, ws + fl.x.codes, ws + fl.x.sf, rxt, sv + sl.xt.codes,
+                                   sv + sl.xt.sf, NVFP4_SF_SWIZZLED_128x4, cuda_stream))
     return st;
   return nvfp4_gemm(ws + fl.x.codes, ws + fl.x.sf, g_x, ws + fl.w.codes, ws + fl.w.sf, g_w, M, N, K, Y, y_dtype, N,
                     cuda_stream);
@@ -166,7 +178,9 @@ extern "C" int nvfp4_linear_bwd_saved(const void* dY, int dtype, int64_t M, int6
   const uint8_t* sv = static_cast<const uint8_t*>(saved);
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   const float* g_dy;
-  if (int st = resolve_g(gscale_mode, dY, dtype, M, N, gdy, reinterpret_cast<float*>(ws + bl.gdy), cuda_stream, &g_dy)) return st;
+  unsigned int* scratch = reinterpret_cast<unsigned int*>(ws + bl.scratch);
+  if (int st = zero_scratch(gscale_mode, scratch, cuda_stream)) return st;
+  if (int st = resolve_g(gscale_mode, dY, dtype, M, N, gdy, reinterpret_cast<float*>(ws + bl.gdy), scratch, cuda_stream, &g_dy)) return st;
   const bool scaled = gscale_mode != NVFP4_G_NONE;     // must match the mode nvfp4_linear_fwd_save ran with
   const float* g_x = scaled ? reinterpret_cast<const float*>(sv + sl.gx) : nullptr;
   const float* g_w = scaled ? reinterpret_cast<const float*>(sv + sl.gw) : nullptr;
@@ -187,9 +201,11 @@ extern "C" int nvfp4_linear_bwd(const void* dY, const void* W, const void* X, in
   if (!buffer_ok(workspace, workspace_bytes, bl.total)) return NVFP4_ERR_WORKSPACE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   const float *g_dy, *g_w, *g_x;
-  if (int st = resolve_g(gscale_mode, dY, dtype, M, N, gdy, reinterpret_cast<float*>(ws + bl.gdy), cuda_stream, &g_dy)) return st;
-  if (int st = resolve_g(gscale_mode, W, dtype, N, K, gw, reinterpret_cast<float*>(ws + bl.gw), cuda_stream, &g_w)) return st;
-  if (int st = resolve_g(gscale_mode, X, dtype, M, K, gx, reinterpret_cast<float*>(ws + bl.gx), cuda_stream, &g_x)) return st;
+  unsigned int* scratch = reinterpret_cast<unsigned int*>(ws + bl.scratch);
+  if (int st = zero_scratch(gscale_mode, scratch, cuda_stream)) return st;
+  if (int st = resolve_g(gscale_mode, dY, dtype, M, N, gdy, reinterpret_cast<float*>(ws + bl.gdy), scratch, cuda_stream, &g_dy)) return st;
+  if (int st = resolve_g(gscale_mode, W, dtype, N, K, gw, reinterpret_cast<float*>(ws + bl.gw), scratch + 2, cuda_stream, &g_w)) return st;
+  if (int st = resolve_g(gscale_mode, X, dtype, M, K, gx, reinterpret_cast<float*>(ws + bl.gx), scratch + 4, cuda_stream, &g_x)) return st;
   if (int st = nvfp4_quantize(W, dtype, N, K, K, 1, g_w, rwt, ws + bl.wt.codes, ws + bl.wt.sf, NVFP4_SF_SWIZZLED_128x4, cuda_stream))
     return st;
   if (int st = nvfp4_quantize(X, dtype, M, K, K, 1, g_x, rxt, ws + bl.xt.codes, ws + bl.xt.sf, NVFP4_SF_SWIZZLED_128x4, cuda_stream))

@@ -305,6 +305,66 @@ __global__ void __launch_bounds__(kThreads) amax_flat_kernel(const uint32_t* x, 
   if ((threadIdx.x & 31) == 0 && amax > 0.0f) atomicMax(out_bits, __float_as_uint(amax));
 }
 
+// The same sweep as one launch: `scratch` = {running max bits, ticket}, both zero on entry.  The block that
+// takes the last ticket turns the maximum into g = amax / 2688 (1 for an all-zero tensor), stores it and
+// leaves the scratch words zero again.
+template <typename T>
+__global__ void __launch_bounds__(kThreads) amax_flat_ticket_kernel(const uint32_t* x, int64_t n_vec32, unsigned int* scratch,
+                                                                    float* g_out) {
+  __shared__ float warp_max[kThreads / 32];
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+  uint32_t mb = 0u;
+  float mf = 0.0f;
+  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec32; i += 4 * stride) {
+    uint32_t w[4][8];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int64_t j = i + u * stride;
+      if (j < n_vec32) {
+        asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                     : "=r"(w[u][0]), "=r"(w[u][1]), "=r"(w[u][2]), "=r"(w[u][3]), "=r"(w[u][4]), "=r"(w[u][5]),
+                       "=r"(w[u][6]), "=r"(w[u][7])
+                     : "l"(x + j * 8));
+      } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) w[u][k] = 0u;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if constexpr (sizeof(T) == 2) {
+        mb = absmax_bf16x2(absmax_bf16x2(absmax_bf16x2(absmax_bf16x2(w[u][0], w[u][1]), absmax_bf16x2(w[u][2], w[u][3])),
+                                         absmax_bf16x2(absmax_bf16x2(w[u][4], w[u][5]), absmax_bf16x2(w[u][6], w[u][7]))),
+                           mb);
+      } else {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) mf = fmaxf(mf, fabsf(__uint_as_float(w[u][k])));
+      }
+    }
+  }
+  float amax = mf;
+  if constexpr (sizeof(T) == 2) {
+    mb &= 0x7FFF7FFFu;
+    amax = fmaxf(__uint_as_float(mb << 16), __uint_as_float(mb & 0xFFFF0000u));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = amax;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int w8 = 1; w8 < kThreads / 32; ++w8) amax = fmaxf(amax, warp_max[w8]);
+    if (amax > 0.0f) atomicMax(&scratch[0], __float_as_uint(amax));      // non-negative floats order as ints
+    __threadfence();
+    if (atomicAdd(&scratch[1], 1u) == gridDim.x - 1) {                    // every other block's maximum is in
+      __threadfence();
+      const float total = __uint_as_float(atomicExch(&scratch[0], 0u));
+      *g_out = (total == 0.0f) ? 1.0f : __fdiv_rn(total, 2688.0f);
+      scratch[1] = 0u;
+    }
+  }
+}
+
 __global__ void amax_finalize_kernel(float* out) {
   const float amax = *out;
   *out = (amax == 0.0f) ? 1.0f : __fdiv_rn(amax, 2688.0f);
@@ -474,6 +534,29 @@ extern "C" int nvfp4_quantize_dual(const void* x, int dtype, int64_t rows, int64
     return st;
   return nvfp4_quantize(x, dtype, rows, cols, ld, 1, global_scale, rounding_t, codes_t, scales_t, sf_layout, cuda_stream);
 }
+
+namespace nvfp4 {
+// Per-tensor scale in one launch where the tensor allows it (dense, 32-byte aligned); `scratch_zeroed` is two
+// zeroed 32-bit words in device memory that the kernel leaves zeroed.  Otherwise the three-step public path.
+int tensor_amax_scale_ws(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld, float* g_out,
+                         unsigned int* scratch_zeroed, void* cuda_stream) {
+  const int64_t total_bytes = rows * cols * (dtype == NVFP4_BF16 ? 2 : 4);
+  if (!x || !g_out || !scratch_zeroed || rows <= 0 || cols <= 0 || ld != cols || (reinterpret_cast<uintptr_t>(x) & 31u) != 0 ||
+      total_bytes % 32 != 0)
+    return nvfp4_tensor_amax_scale(x, dtype, rows, cols, ld, g_out, cuda_stream);
+  if (dtype != NVFP4_BF16 && dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if (int st = check_arch()) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const int64_t n32 = total_bytes / 32;
+  int64_t fb = ceil_div(n32, (int64_t)kThreads * 4);
+  if (fb > 148 * 8) fb = 148 * 8;
+  if (dtype == NVFP4_BF16)
+    amax_flat_ticket_kernel<__nv_bfloat16><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, scratch_zeroed, g_out);
+  else
+    amax_flat_ticket_kernel<float><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, scratch_zeroed, g_out);
+  return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+}  // namespace nvfp4
 
 extern "C" int nvfp4_tensor_amax_scale(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
                                        float* global_scale_out, void* cuda_stream) {
