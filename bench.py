@@ -28,9 +28,9 @@ METRIC = "NVFP4 linear fwd+bwd TFLOPS (% FP4 peak); quantizer GB/s (% HBM peak)"
 FP4_OVER_BF16 = 4.0        # nominal dense ratio: 9 PFLOP/s NVFP4 vs 2.25 PFLOP/s bf16
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic of the GEMM kernel from the committed ncu capture (profiles/gemm2_nvfp4_kernel_8192x8192x4096.md):
-# 83.3 MB read + 211.5 MB written for 306.2 MB of algorithmic bytes (operand codes and scales + fp32 output).
+# 83.0 MB read + 212.2 MB written for 306.2 MB of algorithmic bytes (operand codes and scales + fp32 output).
 # GEMM traffic follows bytes, not FLOPs, so the workload's figure is this ratio times its own algorithmic bytes.
-GEMM_TRAFFIC_RATIO = (83.28 + 211.53) / 306.2
+GEMM_TRAFFIC_RATIO = (83.05 + 212.17) / 306.2
 
 
 def load_peaks():
