@@ -60,9 +60,16 @@ typedef enum { NVFP4_LINEAR_FWD = 0, NVFP4_LINEAR_BWD_DX = 1, NVFP4_LINEAR_BWD_D
 
 /* Rounding of one operand, chosen per call (Eq. 4-6 fix the paper's choice per
  * site; any site may be overridden, as the paper's per-site ablation does).
- * For NVFP4_SR the random byte of element j of block B (B = r*(Kq/16) + kb in
- * the quantized shape) is byte j of Philox4x32-10 with key = seed and counter =
- * (B, offset); the same (seed, offset) reproduces the same codes. */
+ * For NVFP4_SR (Section 1: round to one of the two neighbouring grid values with
+ * probability given by the distance) an element whose scaled magnitude sits at
+ * fraction f of its grid step is rounded up iff floor(f * 2^16) + r >= 2^16 for
+ * a 16-bit random integer r.  Block B (B = r*(Kq/16) + kb in the quantized
+ * shape) draws one Philox4x32-10 output with key = seed and counter =
+ * (B lo, B hi, offset lo, offset hi); output word q (bytes b0..b3, b0 lowest)
+ * serves elements 4q..4q+3: element 4q gets r = b2:b0 (b2 the high byte),
+ * element 4q+1 the same 16 bits in mirrored order, element 4q+2 gets b3:b1 and
+ * element 4q+3 those mirrored.  The same (seed, offset) reproduces the same
+ * codes; distinct offsets give independent streams. */
 typedef struct {
   int32_t mode;      /* nvfp4_round_mode */
   int32_t reserved;  /* must be 0 */
@@ -129,7 +136,12 @@ NVFP4_API int nvfp4_quantization_noise(const void* x, int dtype, int64_t rows, i
 
 /* Per-tensor scale g = max|x| / (6*448), or 1.0f for an all-zero tensor, written
  * to *global_scale_out (device).  The paper defines only the block scale; this
- * optional factor keeps small-magnitude gradients inside the E4M3 scale range. */
+ * optional factor keeps small-magnitude gradients inside the E4M3 scale range.
+ * Non-finite inputs propagate: a tensor that holds a NaN gets g = NaN, one that
+ * holds an infinity (and no NaN) gets g = +Inf, and every element of a product
+ * computed with such a scale (nvfp4_gemm, nvfp4_linear_*) is NaN, so a diverged
+ * step shows in the results.  (With g supplied by the caller, or none, the codes
+ * of a block that holds a non-finite value are unspecified.) */
 NVFP4_API int nvfp4_tensor_amax_scale(const void* x, int dtype, int64_t rows, int64_t cols, int64_t ld,
                             float* global_scale_out, void* cuda_stream);
 
@@ -164,14 +176,18 @@ NVFP4_API int nvfp4_gemm_quantized(const uint8_t* a_codes, const uint8_t* a_sf, 
                          const float* out_global_scale, const nvfp4_rounding* rounding /* host */,
                          uint8_t* out_codes, uint8_t* out_scales, int sf_layout, void* cuda_stream);
 
-/* Tuning/testing hook: force the GEMM kernel variant.  0 restores the automatic
- * choice; 128 / 256 select the single-CTA kernel with a 128 x {128,256} tile;
- * 2128 / 2192 / 2256 select the CTA-pair kernel with a 256 x {128,192,256} tile.
- * Process-wide, not thread-safe. */
+/* TEST HOOK, not part of the supported surface: forces the GEMM kernel variant so
+ * that the tests can compare the library's independent kernel implementations
+ * with each other.  0 restores the automatic choice; 128 / 256 select the
+ * single-CTA kernel with a 128 x {128,256} tile; 2128 / 2192 / 2256 select the
+ * CTA-pair kernel with a 256 x {128,192,256} tile.  Process-wide and
+ * unsynchronised: do not call it while another thread is inside nvfp4_gemm. */
 NVFP4_API int nvfp4_gemm_set_tile_n(int bn);
 
 /* Scratch bytes nvfp4_linear_* needs for a layer of shape (M, N, K);
- * `which` is an nvfp4_linear_kind.  Returns 0 on bad arguments. */
+ * `which` is an nvfp4_linear_kind.  Returns 0 for a layer the calls reject
+ * (non-positive size, contraction length not a multiple of 32, or a contiguous
+ * axis of an operand or of the output not a multiple of 8). */
 NVFP4_API size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int which);
 
 /*

@@ -40,6 +40,8 @@ def lib():
         L.nvfp4o_round_rtn.argtypes = [C.c_float]
         L.nvfp4o_round_sr.restype = C.c_uint8
         L.nvfp4o_round_sr.argtypes = [C.c_float, C.c_uint16]
+        L.nvfp4o_round_sr_many.restype = None
+        L.nvfp4o_round_sr_many.argtypes = [C.c_float, _u16p, C.c_int64, _u8p]
         q = [_f32p, C.c_int64, C.c_int64, C.c_float, C.c_int, C.c_uint64, C.c_uint64, _u8p, _u8p, C.c_int]
         L.nvfp4o_quantize.restype = None
         L.nvfp4o_quantize.argtypes = q
@@ -74,7 +76,7 @@ def lib():
         L.nvfp4o_gemm_f32acc.restype = None
         L.nvfp4o_gemm_f32acc.argtypes = g + [_f32p, C.c_int]
         L.nvfp4o_gemm_sampled.restype = None
-        L.nvfp4o_gemm_sampled.argtypes = g + [_i64p, _i64p, C.c_int64, _f32p, _f32p]
+        L.nvfp4o_gemm_sampled.argtypes = g + [_i64p, _i64p, C.c_int64, _f32p, _f32p, C.c_int]
         L.nvfp4o_sf_swizzled_offset.restype = C.c_int64
         L.nvfp4o_sf_swizzled_offset.argtypes = [C.c_int64, C.c_int64, C.c_int64]
         L.nvfp4o_sf_swizzled_bytes.restype = C.c_int64
@@ -132,6 +134,13 @@ def round_rtn(y: float) -> int:
 
 def round_sr(y: float, r16: int) -> int:
     return int(lib().nvfp4o_round_sr(float(np.float32(y)), r16))
+
+
+def round_sr_many(y: float, r16) -> np.ndarray:
+    r16 = np.ascontiguousarray(r16, dtype=np.uint16)
+    out = np.zeros(r16.size, dtype=np.uint8)
+    lib().nvfp4o_round_sr_many(float(np.float32(y)), r16, r16.size, out)
+    return out
 
 
 def quantize(x, g=1.0, mode=RTN, seed=0, offset=0, transposed=False, nthreads=None):
@@ -260,7 +269,7 @@ def gemm_f32acc(a_codes, a_sf, ga, b_codes, b_sf, gb, nthreads=None):
     return D
 
 
-def gemm_sampled(a_codes, a_sf, ga, b_codes, b_sf, gb, ii, jj):
+def gemm_sampled(a_codes, a_sf, ga, b_codes, b_sf, gb, ii, jj, nthreads=None):
     M, K = a_codes.shape[0], a_codes.shape[1] * 2
     N = b_codes.shape[0]
     ii = np.ascontiguousarray(ii, dtype=np.int64)
@@ -269,7 +278,7 @@ def gemm_sampled(a_codes, a_sf, ga, b_codes, b_sf, gb, ii, jj):
     T = np.zeros(ii.size, dtype=np.float32)
     lib().nvfp4o_gemm_sampled(np.ascontiguousarray(a_codes), np.ascontiguousarray(a_sf), float(np.float32(ga)),
                               np.ascontiguousarray(b_codes), np.ascontiguousarray(b_sf), float(np.float32(gb)),
-                              M, N, K, ii, jj, ii.size, D, T)
+                              M, N, K, ii, jj, ii.size, D, T, host_threads() if nthreads is None else nthreads)
     return D, T
 
 

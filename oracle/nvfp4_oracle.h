@@ -29,7 +29,7 @@ extern "C" {
  * 4-bit pattern s|ee|m in the low nibble. */
 float nvfp4o_e2m1_decode(uint8_t code);
 
-/* Section 3 ("E4M3 format for storing scales"), sign bit unused: unsigned E4M3,
+/* Section 3 (block scales are stored in E4M3), sign bit unused: unsigned E4M3,
  * bias 7, 3 mantissa bits, subnormals, largest finite 448 (0x7E), no infinity.
  * Encode rounds to nearest, ties to the even mantissa, and saturates at 448. */
 uint8_t nvfp4o_e4m3_encode(float v);
@@ -55,6 +55,8 @@ void nvfp4o_block_random_u16(uint64_t seed, uint64_t offset, uint64_t block, uin
  * Both return the 3-bit magnitude code. */
 uint8_t nvfp4o_round_rtn(float y);
 uint8_t nvfp4o_round_sr(float y, uint16_t r16);
+/* nvfp4o_round_sr of one value for n random integers (a loop over the call above). */
+void nvfp4o_round_sr_many(float y, const uint16_t* r16, int64_t n, uint8_t* out);
 
 /* Quantize a logical [Rq, Kq] fp32 tensor (row stride Kq) in blocks of 16 along
  * Kq.  mode 0 = RtN, 1 = SR.  codes: Rq*Kq/2 bytes (element 2i in the low
@@ -107,7 +109,8 @@ void nvfp4o_noise_sums(const float* x, const uint8_t* codes, const uint8_t* scal
  * (unquantized) operands, double accumulation, rounded to fp32; T = sum |a_k b_k|. */
 void nvfp4o_matmul_nt(const float* A, const float* B, int64_t M, int64_t N, int64_t K, float* D, float* T, int nthreads);
 
-/* g = amax / (6*448) in one fp32 division, 1.0f when amax == 0. */
+/* g = amax / (6*448) in one fp32 division, 1.0f when amax == 0.  Non-finite inputs propagate:
+ * NaN if any element is NaN, else +Inf if any element is infinite. */
 float nvfp4o_tensor_amax_scale(const float* x, int64_t n);
 
 /* D[i,j] = (gA*gB) * sum_kb sA[i,kb]*sB[j,kb] * sum_{k in kb} a[i,k]*b[j,k]
@@ -129,7 +132,7 @@ void nvfp4o_gemm_sampled(const uint8_t* a_codes, const uint8_t* a_sf, float ga,
                          const uint8_t* b_codes, const uint8_t* b_sf, float gb,
                          int64_t M, int64_t N, int64_t K,
                          const int64_t* ii, const int64_t* jj, int64_t n,
-                         float* D, float* T);
+                         float* D, float* T, int nthreads);
 
 /* Scale-factor storage in 128-row x 4-block tiles of 512 bytes (the layout the
  * Blackwell block-scaled MMA consumes): byte offset of scale (r, kb) for a

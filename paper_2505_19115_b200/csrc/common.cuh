@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "nvfp4.h"
+#include "per_device.h"
 
 namespace nvfp4 {
 
@@ -16,6 +17,22 @@ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
 // Checks that the current device is a compute-capability 10.x part (cached per device).
 int check_arch();
+
+// Ordinal of the current device (-1 if the runtime cannot tell) and its multiprocessor count (cached per device).
+int current_device();
+int sm_count();
+
+// Raises the dynamic shared-memory limit of `kernel` to `bytes` on the current device, once per device:
+// the attribute belongs to (function, device), so `flags` is a static of the calling instantiation.
+template <class Kernel>
+inline cudaError_t set_max_dynamic_smem(DeviceFlags& flags, Kernel kernel, int bytes) {
+  cudaError_t err = cudaSuccess;
+  once_per_device(flags, current_device(), [&] {
+    err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return err == cudaSuccess;
+  });
+  return err;
+}
 
 // Tile quantizer (quantize_tile.cu): transposed output, optionally the row output from the same read.
 bool tile_quantizer_eligible(int dtype, int64_t rows, int64_t cols, bool dual);

@@ -1049,16 +1049,6 @@ bool make_out_map(CUtensorMap* map, void* base, int64_t M, int64_t N, int64_t ld
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int sm_count() {
-  static int n = 0;
-  if (!n) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
-}
-
 template <int BN>
 int launch_gemm(const uint8_t* a_codes, const uint8_t* b_codes, GemmParams p, cudaStream_t s) {
   using C = Cfg<BN>;
@@ -1067,12 +1057,8 @@ int launch_gemm(const uint8_t* a_codes, const uint8_t* b_codes, GemmParams p, cu
   if (!make_codes_map(&map_b, b_codes, p.N, p.K / 2, BN)) return NVFP4_ERR_CUDA;
   p.tiles_m = (p.M + BM - 1) / BM;
   p.tiles_n = (p.N + BN - 1) / BN;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm_nvfp4_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-      return NVFP4_ERR_CUDA;
-    attr_set = true;
-  }
+  static DeviceFlags smem_set;                         // per instantiation, per device
+  if (set_max_dynamic_smem(smem_set, gemm_nvfp4_kernel<BN>, C::kSmemBytes) != cudaSuccess) return NVFP4_ERR_CUDA;
   const int tiles = p.tiles_m * p.tiles_n;
   const int grid = tiles < sm_count() ? tiles : sm_count();
   gemm_nvfp4_kernel<BN><<<grid, kGemmThreads, C::kSmemBytes, s>>>(map_a, map_b, p);
@@ -1131,13 +1117,9 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
   p.out_nkb = g.N / 16; p.out_k_tiles = ceil_div(p.out_nkb, 4);
   philox_stream_init(&p.out_rng, q.rounding ? q.rounding->seed : 0, q.rounding ? q.rounding->offset : 0);
   if (q.rounding) p.out_sr = q.rounding->mode == NVFP4_SR;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(gemm2_nvfp4_kernel<BN, OUT, BF16_IN, MX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             C::kSmemBytes) != cudaSuccess)
-      return NVFP4_ERR_CUDA;
-    attr_set = true;
-  }
+  static DeviceFlags smem_set;                         // per instantiation, per device
+  if (set_max_dynamic_smem(smem_set, gemm2_nvfp4_kernel<BN, OUT, BF16_IN, MX>, C::kSmemBytes) != cudaSuccess)
+    return NVFP4_ERR_CUDA;
   const int tiles = p.tiles_m * p.tiles_n;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;

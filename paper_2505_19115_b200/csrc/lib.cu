@@ -15,6 +15,20 @@ int check_arch() {
   return ok ? NVFP4_OK : NVFP4_ERR_ARCH;
 }
 
+int current_device() {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
+
+int sm_count() {
+  static DeviceInts table;
+  const int dev = current_device();
+  return cached_per_device(table, dev, 148, [&] {
+    int n = 0;
+    return (dev >= 0 && cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess) ? n : 0;
+  });
+}
+
 }  // namespace nvfp4
 
 extern "C" const char* nvfp4_status_string(int status) {

@@ -25,6 +25,12 @@ bool make_plan(int64_t M, int64_t N, int64_t K, int which, Plan* pl) {
   }
 }
 
+// The shapes the layer calls take (the same predicate sizes the workspace): code rows of K/2 bytes need a
+// 16-byte pitch for the tiled copies, source rows and output rows are moved in 16-byte pieces.
+bool plan_ok(const Plan& pl) {
+  return pl.gemm_k % 32 == 0 && pl.a_cols % 8 == 0 && pl.b_cols % 8 == 0 && pl.gemm_n % 8 == 0;
+}
+
 inline size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
 struct Layout {
@@ -55,8 +61,7 @@ int run_linear(int which, const void* a, const void* b, int dtype, int64_t M, in
   if (gscale_mode == NVFP4_G_GIVEN && (!ga || !gb)) return NVFP4_ERR_NULL;
   Plan pl;
   if (!make_plan(M, N, K, which, &pl)) return NVFP4_ERR_SHAPE;
-  if (pl.gemm_k % 32 != 0) return NVFP4_ERR_SHAPE;
-  if (pl.a_cols % 8 != 0 || pl.b_cols % 8 != 0 || pl.gemm_n % 8 != 0) return NVFP4_ERR_SHAPE;
+  if (!plan_ok(pl)) return NVFP4_ERR_SHAPE;
   const Layout l = make_layout(pl);
   if (!workspace || workspace_bytes < l.total || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return NVFP4_ERR_WORKSPACE;
 
@@ -88,7 +93,7 @@ using namespace nvfp4;
 
 extern "C" size_t nvfp4_linear_workspace_bytes(int64_t M, int64_t N, int64_t K, int which) {
   Plan pl;
-  if (!make_plan(M, N, K, which, &pl) || pl.gemm_k % 16 != 0) return 0;
+  if (!make_plan(M, N, K, which, &pl) || !plan_ok(pl)) return 0;
   return make_layout(pl).total;
 }
 

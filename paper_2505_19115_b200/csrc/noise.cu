@@ -123,7 +123,7 @@ extern "C" int nvfp4_quantization_noise(const void* x, int dtype, int64_t rows, 
   p.codes = codes; p.scales = scales; p.nkb = Kq / 16; p.k_tiles = ceil_div(p.nkb, 4);
   p.swizzled = sf_layout == NVFP4_SF_SWIZZLED_128x4; p.sums = sums;
   int64_t blocks = ceil_div(rows * (cols / 8), (int64_t)kNoiseThreads * 4);
-  if (blocks > 148 * 8) blocks = 148 * 8;
+  if (blocks > sm_count() * 8) blocks = sm_count() * 8;
   if (blocks < 1) blocks = 1;
   if (dtype == NVFP4_BF16) noise_kernel<__nv_bfloat16><<<(unsigned)blocks, kNoiseThreads, 0, s>>>(p);
   else noise_kernel<float><<<(unsigned)blocks, kNoiseThreads, 0, s>>>(p);

@@ -238,36 +238,79 @@ __global__ void __launch_bounds__(kThreads, 3) quantize_transposed_kernel(const 
 
 // -------------------------------------------------------------------------------------------------
 // Per-tensor amax -> g = amax / (6*448)
+//
+// The running maximum is kept as the bit pattern of |x|: non-negative IEEE patterns order as unsigned
+// integers, +Inf sits above every finite value and every NaN pattern above +Inf.  A tensor that
+// holds a NaN therefore gets g = NaN, one that holds an infinity (and no NaN) g = +Inf, and every
+// product computed with such a scale comes out as NaN (NaN * acc, or Inf * 0): a diverged step is
+// visible in Y, dX and dW instead of being quantized into finite codes.
 // -------------------------------------------------------------------------------------------------
+// max |.| of two packed bf16 pairs, per half, NaN if either is (the sign bits of the result are meaningless)
+__device__ __forceinline__ uint32_t absmax_nan_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t r;
+  asm("max.NaN.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(b));
+  return r;
+}
+
+// Running maximum of one thread over words of source data (bf16 pairs or fp32 values).
+template <typename T>
+struct AmaxBits {
+  uint32_t m = 0u;
+  __device__ __forceinline__ void add8(const uint32_t (&w)[8]) {
+    if constexpr (sizeof(T) == 2) {
+      m = absmax_nan_bf16x2(absmax_nan_bf16x2(absmax_nan_bf16x2(absmax_nan_bf16x2(w[0], w[1]), absmax_nan_bf16x2(w[2], w[3])),
+                                              absmax_nan_bf16x2(absmax_nan_bf16x2(w[4], w[5]), absmax_nan_bf16x2(w[6], w[7]))),
+                            m);
+    } else {
+#pragma unroll
+      for (int k = 0; k < 8; ++k) m = max(m, w[k] & 0x7FFFFFFFu);
+    }
+  }
+  __device__ __forceinline__ void add4(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    if constexpr (sizeof(T) == 2) {
+      m = absmax_nan_bf16x2(absmax_nan_bf16x2(absmax_nan_bf16x2(a, b), absmax_nan_bf16x2(c, d)), m);
+    } else {
+      m = max(max(m, a & 0x7FFFFFFFu), max(max(b & 0x7FFFFFFFu, c & 0x7FFFFFFFu), d & 0x7FFFFFFFu));
+    }
+  }
+  // fp32 bit pattern of the maximum over the warp
+  __device__ __forceinline__ uint32_t warp_bits() const {
+    uint32_t bits = m;
+    if constexpr (sizeof(T) == 2) {
+      const uint32_t h = m & 0x7FFF7FFFu;                      // bf16 patterns widen to fp32 by a shift
+      bits = max(h >> 16, h & 0xFFFFu) << 16;
+    }
+    return __reduce_max_sync(0xFFFFFFFFu, bits);
+  }
+};
+
+// Strided tensors: 16-byte loads, grid-stride.
 template <typename T>
 __global__ void __launch_bounds__(kThreads) amax_kernel(const T* x, int64_t rows, int64_t cols, int64_t ld,
                                                         unsigned int* out_bits) {
   constexpr int kVec = 16 / (int)sizeof(T);
   const int64_t vec_per_row = cols / kVec;
   const int64_t total = rows * vec_per_row;
-  float amax = 0.0f;
+  AmaxBits<T> acc;
   for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < total; i += (int64_t)gridDim.x * kThreads) {
     const int64_t r = i / vec_per_row, vcol = i % vec_per_row;
     const uint4 q = __ldg(reinterpret_cast<const uint4*>(x + r * ld + vcol * kVec));
-    if constexpr (sizeof(T) == 2) {
-      const uint32_t m = absmax_bf16x2(absmax_bf16x2(q.x, q.y), absmax_bf16x2(q.z, q.w)) & 0x7FFF7FFFu;
-      amax = fmaxf(amax, fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u)));
-    } else {
-      amax = fmaxf(fmaxf(fabsf(__uint_as_float(q.x)), fabsf(__uint_as_float(q.y))),
-                   fmaxf(fmaxf(fabsf(__uint_as_float(q.z)), fabsf(__uint_as_float(q.w))), amax));
-    }
+    acc.add4(q.x, q.y, q.z, q.w);
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
-  if ((threadIdx.x & 31) == 0 && amax > 0.0f) atomicMax(out_bits, __float_as_uint(amax));  // non-negative floats order as ints
+  const uint32_t bits = acc.warp_bits();
+  if ((threadIdx.x & 31) == 0 && bits != 0u) atomicMax(out_bits, bits);
 }
 
 // Dense tensors (ld == cols, 32-byte aligned): a flat sweep with four 256-bit loads in flight per thread.
-template <typename T>
-__global__ void __launch_bounds__(kThreads) amax_flat_kernel(const uint32_t* x, int64_t n_vec32, unsigned int* out_bits) {
+// TICKET = false: the maximum is left in out[0] for amax_finalize_kernel.
+// TICKET = true: one launch does it all.  out = {running max bits, ticket}, both zero on entry; the block that
+// takes the last ticket turns the maximum into g = amax / 2688 (1 for an all-zero tensor), stores it in *g_out
+// and leaves the two words zero again.
+template <typename T, bool TICKET>
+__global__ void __launch_bounds__(kThreads) amax_flat_kernel(const uint32_t* x, int64_t n_vec32, unsigned int* out, float* g_out) {
+  __shared__ uint32_t warp_max[kThreads / 32];
   const int64_t stride = (int64_t)gridDim.x * kThreads;
-  uint32_t mb = 0u;        // bf16: packed running |max| pair
-  float mf = 0.0f;         // fp32: running max
+  AmaxBits<T> acc;
   for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec32; i += 4 * stride) {
     uint32_t w[4][8];
 #pragma unroll
@@ -284,83 +327,26 @@ __global__ void __launch_bounds__(kThreads) amax_flat_kernel(const uint32_t* x, 
       }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if constexpr (sizeof(T) == 2) {
-        mb = absmax_bf16x2(absmax_bf16x2(absmax_bf16x2(absmax_bf16x2(w[u][0], w[u][1]), absmax_bf16x2(w[u][2], w[u][3])),
-                                         absmax_bf16x2(absmax_bf16x2(w[u][4], w[u][5]), absmax_bf16x2(w[u][6], w[u][7]))),
-                           mb);
-      } else {
-#pragma unroll
-        for (int k = 0; k < 8; ++k) mf = fmaxf(mf, fabsf(__uint_as_float(w[u][k])));
-      }
-    }
+    for (int u = 0; u < 4; ++u) acc.add8(w[u]);
   }
-  float amax = mf;
-  if constexpr (sizeof(T) == 2) {
-    mb &= 0x7FFF7FFFu;
-    amax = fmaxf(__uint_as_float(mb << 16), __uint_as_float(mb & 0xFFFF0000u));
-  }
+  const uint32_t bits = acc.warp_bits();
+  if constexpr (!TICKET) {
+    if ((threadIdx.x & 31) == 0 && bits != 0u) atomicMax(out, bits);
+  } else {
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = bits;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t block_bits = bits;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
-  if ((threadIdx.x & 31) == 0 && amax > 0.0f) atomicMax(out_bits, __float_as_uint(amax));
-}
-
-// The same sweep as one launch: `scratch` = {running max bits, ticket}, both zero on entry.  The block that
-// takes the last ticket turns the maximum into g = amax / 2688 (1 for an all-zero tensor), stores it and
-// leaves the scratch words zero again.
-template <typename T>
-__global__ void __launch_bounds__(kThreads) amax_flat_ticket_kernel(const uint32_t* x, int64_t n_vec32, unsigned int* scratch,
-                                                                    float* g_out) {
-  __shared__ float warp_max[kThreads / 32];
-  const int64_t stride = (int64_t)gridDim.x * kThreads;
-  uint32_t mb = 0u;
-  float mf = 0.0f;
-  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < n_vec32; i += 4 * stride) {
-    uint32_t w[4][8];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int64_t j = i + u * stride;
-      if (j < n_vec32) {
-        asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                     : "=r"(w[u][0]), "=r"(w[u][1]), "=r"(w[u][2]), "=r"(w[u][3]), "=r"(w[u][4]), "=r"(w[u][5]),
-                       "=r"(w[u][6]), "=r"(w[u][7])
-                     : "l"(x + j * 8));
-      } else {
-#pragma unroll
-        for (int k = 0; k < 8; ++k) w[u][k] = 0u;
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      if constexpr (sizeof(T) == 2) {
-        mb = absmax_bf16x2(absmax_bf16x2(absmax_bf16x2(absmax_bf16x2(w[u][0], w[u][1]), absmax_bf16x2(w[u][2], w[u][3])),
-                                         absmax_bf16x2(absmax_bf16x2(w[u][4], w[u][5]), absmax_bf16x2(w[u][6], w[u][7]))),
-                           mb);
-      } else {
-#pragma unroll
-        for (int k = 0; k < 8; ++k) mf = fmaxf(mf, fabsf(__uint_as_float(w[u][k])));
-      }
-    }
-  }
-  float amax = mf;
-  if constexpr (sizeof(T) == 2) {
-    mb &= 0x7FFF7FFFu;
-    amax = fmaxf(__uint_as_float(mb << 16), __uint_as_float(mb & 0xFFFF0000u));
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
-  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = amax;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-#pragma unroll
-    for (int w8 = 1; w8 < kThreads / 32; ++w8) amax = fmaxf(amax, warp_max[w8]);
-    if (amax > 0.0f) atomicMax(&scratch[0], __float_as_uint(amax));      // non-negative floats order as ints
-    __threadfence();
-    if (atomicAdd(&scratch[1], 1u) == gridDim.x - 1) {                    // every other block's maximum is in
+      for (int w8 = 1; w8 < kThreads / 32; ++w8) block_bits = max(block_bits, warp_max[w8]);
+      if (block_bits != 0u) atomicMax(&out[0], block_bits);
       __threadfence();
-      const float total = __uint_as_float(atomicExch(&scratch[0], 0u));
-      *g_out = (total == 0.0f) ? 1.0f : __fdiv_rn(total, 2688.0f);
-      scratch[1] = 0u;
+      if (atomicAdd(&out[1], 1u) == gridDim.x - 1) {                      // every other block's maximum is in
+        __threadfence();
+        const float total = __uint_as_float(atomicExch(&out[0], 0u));
+        *g_out = (total == 0.0f) ? 1.0f : __fdiv_rn(total, 2688.0f);
+        out[1] = 0u;
+      }
     }
   }
 }
@@ -381,13 +367,8 @@ template <typename T, bool SR, bool SWZ>
 cudaError_t launch_transposed(const QuantParams& p, cudaStream_t s) {
   using TT = TTile<T>;
   const size_t smem = TT::kRows * kTCols * sizeof(T) + kTCols * TT::kCodePitch + kTCols * TT::kRowBlocks;
-  static bool attr_set = false;  // one attribute per instantiation; harmless if repeated
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(quantize_transposed_kernel<T, SR, SWZ>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static DeviceFlags smem_set;   // per instantiation, per device
+  if (cudaError_t e = set_max_dynamic_smem(smem_set, quantize_transposed_kernel<T, SR, SWZ>, (int)smem)) return e;
   dim3 grid((unsigned)ceil_div(p.cols, kTCols), (unsigned)ceil_div(p.rows, TT::kRows));
   quantize_transposed_kernel<T, SR, SWZ><<<grid, kThreads, smem, s>>>(p);
   return cudaGetLastError();
@@ -549,11 +530,11 @@ int tensor_amax_scale_ws(const void* x, int dtype, int64_t rows, int64_t cols, i
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const int64_t n32 = total_bytes / 32;
   int64_t fb = ceil_div(n32, (int64_t)kThreads * 4);
-  if (fb > 148 * 8) fb = 148 * 8;
+  if (fb > sm_count() * 8) fb = sm_count() * 8;
   if (dtype == NVFP4_BF16)
-    amax_flat_ticket_kernel<__nv_bfloat16><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, scratch_zeroed, g_out);
+    amax_flat_kernel<__nv_bfloat16, true><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, scratch_zeroed, g_out);
   else
-    amax_flat_ticket_kernel<float><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, scratch_zeroed, g_out);
+    amax_flat_kernel<float, true><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, scratch_zeroed, g_out);
   return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 }  // namespace nvfp4
@@ -569,18 +550,18 @@ extern "C" int nvfp4_tensor_amax_scale(const void* x, int dtype, int64_t rows, i
   if (cudaMemsetAsync(global_scale_out, 0, sizeof(float), s) != cudaSuccess) return NVFP4_ERR_CUDA;
   const int64_t vecs = rows * (cols / (dtype == NVFP4_BF16 ? 8 : 4));
   int64_t blocks = ceil_div(vecs, (int64_t)kThreads * 4);
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
   if (blocks < 1) blocks = 1;
   unsigned int* bits = reinterpret_cast<unsigned int*>(global_scale_out);
   const int64_t total_bytes = rows * cols * (dtype == NVFP4_BF16 ? 2 : 4);
   if (ld == cols && (reinterpret_cast<uintptr_t>(x) & 31u) == 0 && total_bytes % 32 == 0) {
     const int64_t n32 = total_bytes / 32;
     int64_t fb = ceil_div(n32, (int64_t)kThreads * 4);
-    if (fb > 148 * 8) fb = 148 * 8;
+    if (fb > sm_count() * 8) fb = sm_count() * 8;
     if (dtype == NVFP4_BF16)
-      amax_flat_kernel<__nv_bfloat16><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, bits);
+      amax_flat_kernel<__nv_bfloat16, false><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, bits, nullptr);
     else
-      amax_flat_kernel<float><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, bits);
+      amax_flat_kernel<float, false><<<(unsigned)fb, kThreads, 0, s>>>(static_cast<const uint32_t*>(x), n32, bits, nullptr);
   } else if (dtype == NVFP4_BF16)
     amax_kernel<__nv_bfloat16><<<(unsigned)blocks, kThreads, 0, s>>>(static_cast<const __nv_bfloat16*>(x), rows, cols, ld, bits);
   else

@@ -214,13 +214,8 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* base, uin
 template <bool SR_T, bool DUAL, bool SR_R, bool SWZ>
 cudaError_t launch_tile(const CUtensorMap& mx, const CUtensorMap& mct, const CUtensorMap& mcr, const TileParams& p,
                         cudaStream_t s) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(quantize_tile_kernel<SR_T, DUAL, SR_R, SWZ>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kTileSmem);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static DeviceFlags smem_set;   // per instantiation, per device
+  if (cudaError_t e = set_max_dynamic_smem(smem_set, quantize_tile_kernel<SR_T, DUAL, SR_R, SWZ>, kTileSmem)) return e;
   dim3 grid((unsigned)ceil_div(p.cols, kTileCols), (unsigned)ceil_div(p.rows, kTileRows));
   quantize_tile_kernel<SR_T, DUAL, SR_R, SWZ><<<grid, kThreads, kTileSmem, s>>>(mx, mct, mcr, p);
   return cudaGetLastError();

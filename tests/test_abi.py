@@ -47,6 +47,21 @@ def test_workspace_bytes():
         assert n > 0 and n % 256 == 0
     assert nb.nvfp4_linear_workspace_bytes(256, 512, 512, 5) == 0
     assert nb.nvfp4_linear_workspace_bytes(0, 512, 512, 0) == 0
+    # the size query refuses exactly the layers the calls refuse: a contraction length that is a multiple
+    # of 16 but not of 32 (K for fwd, N for dx, M for dw), or a contiguous axis that is not a multiple of 8
+    assert nb.nvfp4_linear_workspace_bytes(256, 512, 528, 0) == 0
+    assert nb.nvfp4_linear_workspace_bytes(256, 528, 512, 1) == 0
+    assert nb.nvfp4_linear_workspace_bytes(272, 512, 512, 2) == 0
+    assert nb.nvfp4_linear_workspace_bytes(256, 516, 512, 0) == 0          # Y rows of 516 elements
+    assert nb.nvfp4_linear_workspace_bytes(256, 512, 544, 0) > 0
+
+
+def test_static_forward_rejects_what_the_size_query_rejects():
+    L = nb.lib()
+    r = nb.Rounding()
+    buf = C.c_void_p(0x1000)
+    st = L.nvfp4_linear_fwd_static(buf, buf, 0, 256, 512, 528, 0, None, None, C.byref(r), C.byref(r), buf, 1, None)
+    assert st == 2                                                          # shape error, not a late failure
 
 
 def test_quantize_argument_errors_are_host_side():

@@ -153,3 +153,35 @@ def test_fused_layer_with_given_scales_and_bf16_outputs():
     ref, T = oracle_linear("dx", dY, W, nb.Rounding(nb.SR, 0, 0), rt, True)
     assert np.all(np.abs(_host(dX) - ref) <= TOL * T + np.abs(ref) * 2.0 ** -8)
     _assert_close(_host(dW), *oracle_linear("dw", dY, X, nb.Rounding(nb.SR, 0, 1), nb.Rounding(nb.SR, 0, 2), True))
+
+
+# ---------------------------------------------------------------- non-finite inputs stay visible
+@pytest.mark.parametrize("bad", [float("nan"), float("inf"), float("-inf")])
+def test_non_finite_input_propagates_through_the_per_tensor_scale(bad):
+    # A NaN (or an infinity) anywhere in an operand makes its amax scale NaN (+Inf), as the oracle's does, and
+    # every element of a product computed with that scale NaN; products of the other operands stay finite.
+    M, K, N = 256, 512, 384
+    X, W, dY = synth.linear_inputs(M, K, N, seed=77, grad_std=1e-3)
+    X[131, 257] = bad
+    Xd, Wd, dYd = X.cuda(), W.cuda(), dY.cuda()
+    g = nb.nvfp4_tensor_amax_scale(Xd)
+    want = ob.tensor_amax_scale(_host(Xd))
+    got = float(g.item())
+    assert (np.isnan(want) and np.isnan(got)) or (np.isinf(want) and got == want)
+    for Xin in (Xd, Xd.float()):                        # bf16 and fp32 sources take different amax paths
+        g32 = float(nb.nvfp4_tensor_amax_scale(Xin).item())
+        assert (np.isnan(want) and np.isnan(g32)) or g32 == want
+    Y = nb.nvfp4_linear_fwd(Xd, Wd)
+    dW = nb.nvfp4_linear_bwd_dw(dYd, Xd)
+    dX = nb.nvfp4_linear_bwd_dx(dYd, Wd)
+    Yf, saved = nb.nvfp4_linear_fwd_save(Xd, Wd)
+    dXf, dWf = nb.nvfp4_linear_bwd_saved(dYd, saved, K)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
+    for t in (Y, dW, Yf, dWf):
+        assert bool(torch.isnan(t).all())
+    for t in (dX, dXf):                                 # dX = Q(dY) Q(W^T)^T does not involve X
+        assert bool(torch.isfinite(t).all())
+    # the oracle's dequantize-then-matmul says the same
+    ref, _ = oracle_linear("fwd", Xd, Wd, nb.Rounding(nb.RTN), nb.Rounding(nb.RTN), True)
+    assert np.all(np.isnan(ref))

@@ -228,6 +228,80 @@ def test_sr_neighbouring_elements_round_independently_enough():
     assert abs(both / n - 0.25) < 0.015
 
 
+def test_sr_pair_joint_probability_over_all_random_integers():
+    # The two elements of a pair read the same 16 random bits, one in mirrored order.  For the noise model of
+    # Section 4 / App. B.1 (independent zero-mean errors) their round-up decisions must be close to independent
+    # at every (f0, f1), not only at f = 1/2.  Element 0 rounds up iff r >= 2^16 - F0, which the top byte H of
+    # r decides unless H equals the threshold's top byte (probability 2^-8); element 1 rounds up iff
+    # mirror(r) >= 2^16 - F1, which the mirrored low byte L decides unless it ties (2^-8).  H and L are
+    # independent, and a tie's decision depends on the other byte only through an indicator whose covariance
+    # with the other decision is at most 1/4, so |P(both up) - P0 P1| <= 2 * 2^-8 / 4 + 2^-16.
+    bound = 2.0 ** -9 + 2.0 ** -16
+    rng = np.random.default_rng(11)
+    base = int(rng.integers(0, 2 ** 32))
+    worst = 0.0
+    for pair, (lo_shift, hi_shift) in enumerate(((0, 16), (8, 24))):        # bytes (0, 2) serve elements 0/1, bytes (1, 3) elements 2/3
+        keep = base & ~((0xFF << lo_shift) | (0xFF << hi_shift)) & 0xFFFFFFFF
+        ints = np.array([ob.word_random_u16(keep | ((v & 0xFF) << lo_shift) | ((v >> 8) << hi_shift)) for v in range(65536)],
+                        dtype=np.uint16)
+        r_even, r_odd = ints[:, 2 * pair], ints[:, 2 * pair + 1]
+        assert np.array_equal(np.sort(r_even), np.arange(65536)) and np.array_equal(np.sort(r_odd), np.arange(65536))
+        for _ in range(110):
+            y0, y1 = (np.float32(v) for v in rng.uniform(0.0, 6.0, 2))
+            (lo0, hi0), (lo1, hi1) = _sr_neighbours(float(y0)), _sr_neighbours(float(y1))
+            if lo0 == hi0 or lo1 == hi1:
+                continue
+            up0 = np.array(GRID)[ob.round_sr_many(float(y0), r_even)] == hi0
+            up1 = np.array(GRID)[ob.round_sr_many(float(y1), r_odd)] == hi1
+            d = abs(float(np.mean(up0 & up1)) - float(np.mean(up0)) * float(np.mean(up1)))
+            worst = max(worst, d)
+            assert d <= bound, (pair, float(y0), float(y1), d)
+    assert worst > 0.0                                                       # the pairs are dependent, only weakly
+
+
+def test_sr_errors_of_a_block_behave_like_independent_noise():
+    # 2 * 10^4 seeded draws of one block: the rounding errors of paired elements (0/1, 2/3, ...) are uncorrelated
+    # within 3 sigma, and the variance of the block's summed error equals the sum of the per-element
+    # variances, as independent zero-mean noise would give (App. B.1 assumes E[eps eps^T] = sigma^2 I).
+    x1 = np.array([0.3, -0.7, 1.1, 1.6, 2.2, -2.9, 3.3, 4.7, 5.5, 0.05, 6.0, -0.26, 0.9, 1.9, 3.9, -5.9], dtype=np.float32)
+    n = 20000
+    x = np.tile(x1, (n, 1))                                                  # row r draws block index r
+    codes, scales = ob.quantize(x, mode=ob.SR, seed=123, offset=5)
+    err = ob.dequantize(codes, scales).astype(np.float64) - x.astype(np.float64)
+    sd = err.std(axis=0)
+    assert abs(err.mean(axis=0)).max() <= 3 * sd.max() / np.sqrt(n) + 2.0 / 65536
+    moving = [j for j in range(16) if sd[j] > 0]
+    assert len(moving) >= 14
+    for a in range(0, 16, 2):
+        if sd[a] > 0 and sd[a + 1] > 0:
+            corr = np.mean((err[:, a] - err[:, a].mean()) * (err[:, a + 1] - err[:, a + 1].mean())) / (sd[a] * sd[a + 1])
+            assert abs(corr) <= 3 / np.sqrt(n) + 2.0 ** -7, (a, corr)
+    total = err.sum(axis=1)
+    want = float(np.sum(sd ** 2))
+    # the sample variance of n draws of a sum of bounded terms: relative standard error about sqrt(2/n)
+    assert abs(total.var() - want) <= 4 * np.sqrt(2.0 / n) * want + 0.01 * want
+
+
+def test_tensor_scale_propagates_non_finite_values():
+    # A diverged step must stay visible: NaN anywhere -> NaN, otherwise an infinity -> +Inf.
+    assert np.isnan(ob.tensor_amax_scale(np.array([1.0, np.nan, 3.0], dtype=np.float32)))
+    assert np.isnan(ob.tensor_amax_scale(np.array([np.inf, np.nan], dtype=np.float32)))
+    assert ob.tensor_amax_scale(np.array([1.0, -np.inf], dtype=np.float32)) == np.inf
+    assert ob.tensor_amax_scale(np.array([0.0, 2688.0], dtype=np.float32)) == 1.0
+    # ... and every output of a product computed with such a scale is NaN
+    rng = np.random.default_rng(4)
+    X = rng.standard_normal((8, 64)).astype(np.float32)
+    W = rng.standard_normal((16, 64)).astype(np.float32)
+    for bad in (np.nan, np.inf, -np.inf):
+        Xb = X.copy()
+        Xb[3, 17] = bad
+        gx, gw = ob.tensor_amax_scale(Xb), ob.tensor_amax_scale(W)
+        xc, xs = ob.quantize(Xb, g=gx)
+        wc, ws = ob.quantize(W, g=gw)
+        D, _ = ob.gemm(xc, xs, gx, wc, ws, gw)
+        assert np.all(np.isnan(D)), bad
+
+
 def test_sr_variance_closed_form():
     # y uniform within one grid step: E[err^2] = delta^2/6 under SR, delta^2/12 under RtN
     rng = np.random.default_rng(3)

@@ -49,3 +49,23 @@ def test_layer_beyond_the_fixed_array_is_rejected():
     with pytest.raises(nb.NvFp4Error) as e:
         nb.nvfp4_linear_fwd_static(X, W)
     assert e.value.status == 5
+
+
+def test_the_call_leaves_the_free_device_memory_unchanged():
+    # The property in the entry point's name: with the output preallocated, a call takes no device memory
+    # (cudaMemGetInfo's free bytes are the same before and after).  The first call on a device loads the
+    # kernels and looks up the array's address, so it is made before the measurement.
+    rt = nb.Rounding(nb.RTN)
+    X, W, _ = synth.linear_inputs(256, 512, 512, seed=13)
+    X, W = X.cuda(), W.cuda()
+    out = torch.empty((256, 512), dtype=torch.float32, device="cuda")
+    nb.nvfp4_linear_fwd_static(X, W, rx=rt, rw=rt, out=out)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        nb.nvfp4_linear_fwd_static(X, W, rx=rt, rw=rt, out=out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    want = nb.nvfp4_linear_fwd(X, W, rx=rt, rw=rt)
+    assert torch.equal(out, want)
