@@ -329,6 +329,21 @@ NVFP4_API int nvfp4_linear_fwd_static(const void* X, const void* W, int dtype, i
                                       const nvfp4_rounding* rx, const nvfp4_rounding* rw,
                                       void* Y, int y_dtype, void* cuda_stream);
 
+/*
+ * Measurement aid (the paper has no counterpart): the issue rate of the tensor-core instruction the
+ * GEMM is built on, tcgen05.mma kind::mxf4nvf4 on a CTA pair (256 x instr_n x 64 per instruction; instr_n
+ * a multiple of 32 up to 256, the GEMM uses 256), issued
+ * back to back on operands resident in shared memory and scales resident in tensor memory, one CTA
+ * pair per two multiprocessors, `stages` groups of four instructions each (1 .. 2^20).  No loads and
+ * no epilogue: it gives the ceiling the tensor pipe sets at the clock the run holds, the denominator
+ * of the GEMM's "fraction of issue peak".  out (device, 8-byte aligned, out_bytes >= 24 per pair)
+ * receives per pair {cycles of the leader CTA's clock from first issue to completion, instructions
+ * issued, 1 if the bounded wait for completion ran out}; *pairs_out (host) the number of pairs.
+ * FLOP per instruction: 2 * 256 * instr_n * 64.
+ */
+NVFP4_API int nvfp4_microbench_mma_peak(int stages, int instr_n, int64_t* out, size_t out_bytes,
+                                        int* pairs_out /* host */, void* cuda_stream);
+
 /* Reads and clears the device-side error word of the current device (host
  * out-pointer; synchronises the device).  Non-zero means a kernel gave up on a
  * bounded wait and its output is invalid; bits 0-7 identify the wait site. */

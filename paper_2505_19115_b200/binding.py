@@ -97,6 +97,8 @@ def lib():
     L.nvfp4_linear_bwd_bf16.argtypes = [vp, vp, vp, i64, i64, i64, vp, ci, vp, ci, vp, sz, vp]
     L.nvfp4_linear_fwd_static.restype = ci
     L.nvfp4_linear_fwd_static.argtypes = [vp, vp, ci, i64, i64, i64, ci, vp, vp, rp, rp, vp, ci, vp]
+    L.nvfp4_microbench_mma_peak.restype = ci
+    L.nvfp4_microbench_mma_peak.argtypes = [ci, ci, vp, sz, C.POINTER(C.c_int), vp]
     L.nvfp4_device_error_word.restype = ci
     L.nvfp4_device_error_word.argtypes = [C.POINTER(C.c_uint32)]
     _lib = L
@@ -429,6 +431,17 @@ def nvfp4_linear_fwd_static(X, W, gscale_mode=G_AMAX, gx=None, gw=None, rx=None,
                                        C.byref(rx), C.byref(rw), _ptr(out), _dtype_code(out), _stream(stream))
     _check(st, "nvfp4_linear_fwd_static")
     return out
+
+
+def nvfp4_microbench_mma_peak(stages: int, instr_n: int = 256, device=None, stream=None) -> torch.Tensor:
+    """Issue-rate measurement of the FP4 tensor-core instruction: returns an int64 tensor [pairs, 3] of
+    (cycles, instructions, timed-out flag) per CTA pair."""
+    dev = torch.device("cuda", torch.cuda.current_device()) if device is None else device
+    out = torch.zeros((torch.cuda.get_device_properties(dev).multi_processor_count // 2 + 1, 3), dtype=torch.int64, device=dev)
+    pairs = C.c_int(0)
+    _check(lib().nvfp4_microbench_mma_peak(stages, instr_n, _ptr(out), out.numel() * 8, C.byref(pairs), _stream(stream)),
+           "nvfp4_microbench_mma_peak")
+    return out[:pairs.value]
 
 
 def nvfp4_device_error_word() -> int:

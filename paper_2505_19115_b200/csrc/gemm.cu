@@ -14,12 +14,29 @@
 #include <cuda_bf16.h>
 
 #include "quantize_core.cuh"
+#include "tc_ptx.cuh"
 #include "tensor_map.cuh"
 
 namespace nvfp4 {
 namespace {
 
 __device__ unsigned int g_error_word = 0;
+
+// Cycle account of the CTA-pair kernel (debug builds only: -DNVFP4_GEMM_ACCOUNT, see microbench.py gemm_account).
+// Each role of pair 0 adds up the clock64() cycles it spends in each of its waits and in its work; the product
+// build compiles all of it away.
+#ifdef NVFP4_GEMM_ACCOUNT
+__device__ long long g_account[32];
+#define ACCOUNT_VARS(...) long long __VA_ARGS__
+#define ACCOUNT(var, ...) { const long long acc_t0_ = clock64(); __VA_ARGS__; var += clock64() - acc_t0_; }
+#define ACCOUNT_STORE(cond, slot, value) { if (cond) g_account[slot] = (value); }
+#define ACCOUNT_NOW() clock64()
+#else
+#define ACCOUNT_VARS(...)
+#define ACCOUNT(var, ...) { __VA_ARGS__; }
+#define ACCOUNT_STORE(cond, slot, value)
+#define ACCOUNT_NOW() 0ll
+#endif
 
 constexpr int BM = 128;           // rows of A per tile (= UMMA M)
 constexpr int BK_BYTES = 128;     // packed bytes per row per stage = 256 E2M1 values
@@ -63,33 +80,8 @@ struct GemmParams {
 };
 
 // ------------------------------------------------------------------------------------------------
-// PTX wrappers
+// Bounded waits (the PTX wrappers are in tc_ptx.cuh)
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\t"
-               "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-               "selp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_timer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-
 // Bounded waits.  They return false (and record `site`) if the barrier did not flip within the time
 // limit or another role of this CTA already gave up.
 //
@@ -132,14 +124,6 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
 // memory through the generic proxy: it issues tcgen05.mma, whose shared-memory operands were written
 // by the bulk copies that completed the phase, and whose tensor-memory scales are ordered by
 // tcgen05.fence::after_thread_sync.
-__device__ __forceinline__ bool mbar_try_wait_relaxed(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n\t.reg .pred p;\n\t"
-               "mbarrier.try_wait.parity.relaxed.cta.shared::cta.b64 p, [%1], %2;\n\t"
-               "selp.u32 %0, 1, 0, p;\n\t}"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
 __device__ __forceinline__ bool mbar_wait_issuer(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t site) {
   for (int i = 0; i < 4096; ++i)
     if (mbar_try_wait_relaxed(bar, parity)) return true;
@@ -149,12 +133,6 @@ __device__ __forceinline__ bool mbar_wait_issuer(uint32_t bar, uint32_t parity, 
       if (mbar_try_wait_relaxed(bar, parity)) return true;
     if (mbar_wait_timeout(site, abort_flag, t0)) return false;
   }
-}
-// One lane of a converged warp.
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xFFFFFFFF;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
-  return pred != 0;
 }
 // Whole-warp wait of the scale movers, relaxed polls by every lane: these warps issue tcgen05.st, and
 // next to such operations an acquiring poll costs ~180 cycles even when the phase is complete (see
@@ -171,176 +149,6 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
   ok = __shfl_sync(0xFFFFFFFFu, ok, 0);
   if (ok) (void)mbar_try_wait(bar, parity);
   return ok;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-               ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// 512 bytes of scales (32 rows x 16 bytes in shared memory) -> 4 tensor-memory columns, replicated
-// into all four 32-lane quarters.
-__device__ __forceinline__ void tc_cp_sf(uint32_t taddr, uint64_t sdesc) {
-  asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
-}
-__device__ __forceinline__ void tc_mma_nvf4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                            uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\t"
-               "setp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::1.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// tcgen05.ld fills its registers asynchronously until tcgen05.wait::ld; this empty statement, placed
-// after the wait, makes every later use of the registers depend on it, so the compiler cannot move
-// such a use above the wait.
-__device__ __forceinline__ void tmem_ld_pin(uint32_t (&r)[32]) {
-#pragma unroll
-  for (int i = 0; i < 32; i += 8)
-    asm volatile("" : "+r"(r[i]), "+r"(r[i + 1]), "+r"(r[i + 2]), "+r"(r[i + 3]), "+r"(r[i + 4]), "+r"(r[i + 5]),
-                      "+r"(r[i + 6]), "+r"(r[i + 7]) :: "memory");
-}
-
-// ---- cluster / CTA-pair helpers (cta_group::2 path) ----
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-// Address of the same shared-memory offset in CTA `rank` of this cluster.
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
-  return r;
-}
-// Arrive on a barrier that may live in the peer CTA.  Default semantics (release at CTA scope): a
-// cluster-scope release costs about a thousand cycles here, and the data these arrivals publish
-// lives in tensor memory, whose ordering comes from tcgen05.wait / tcgen05.fence, not from this fence.
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Tiled copy whose completion bytes are signalled on a barrier that may live in the peer CTA.
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t cluster_bar, int x, int y) {
-  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-               ::"r"(dst), "l"(map), "r"(cluster_bar), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t smem_dst, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-// Arrives on the barrier at the same offset in both CTAs of the pair once all prior MMAs finish.
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-               ::"r"(bar), "h"((uint16_t)3) : "memory");
-}
-__device__ __forceinline__ void tc_mma_nvf4_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                                 uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\t"
-               "setp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.scale_vec::4X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
-               : "memory");
-}
-
-// MXFP4: blocks of 32 with UE8M0 scales (two scales per row per instruction)
-__device__ __forceinline__ void tc_mma_mxf4_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                                 uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\t"
-               "setp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
-               : "memory");
-}
-
-// bf16 x bf16 -> fp32, 256 x N x 16 per instruction (the backward / update products of the paper's
-// quantization-aware fine-tuning phase, which run in BF16)
-__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                                 uint32_t accumulate) {
-  asm volatile("{\n\t.reg .pred p;\n\t"
-               "setp.ne.b32 p, %4, 0;\n\t"
-               "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-               ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-// Shared-memory matrix descriptors (64-bit): start address, leading/stride byte offsets (all >> 4),
-// descriptor version 1 at bit 46, swizzle mode at bits 61-63.
-// Operand tiles: K-major, 128-byte swizzle, rows 128 bytes apart, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
-  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
-         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-// Scale tile: 32 rows x 16 bytes, no swizzle, 8-row groups 128 bytes apart.
-__device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
-  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
-}
-// Instruction descriptor of kind::mxf4nvf4: E2M1 x E2M1 (format 1), K-major operands, UE4M3
-// scales, N >> 3 at bit 17, M >> 4 at bit 24.
-// Instruction descriptor of kind::f16 with bf16 operands (format 1) and an fp32 accumulator (bit 4).
-__host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
-// Instruction descriptor of kind::mxf4 (scale_vec::2X): as above with UE8M0 scales (bit 23) and the
-// half of the 32-bit scale column to use (bytes 0-1 or 2-3) at bits 4-5 (B) and 29-30 (A).
-__host__ __device__ constexpr uint32_t instr_desc_mx(int m, int n, int sf_half) {
-  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (1u << 23) | ((uint32_t)(m >> 4) << 24) |
-         ((uint32_t)(2 * sf_half) << 4) | ((uint32_t)(2 * sf_half) << 29);
-}
-__host__ __device__ constexpr uint32_t instr_desc(int m, int n) {
-  return (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | (0u << 23) | ((uint32_t)(m >> 4) << 24);
 }
 
 // Tile order: panels of kPanel row tiles, column-major inside a panel, so that the CTAs running at
@@ -673,12 +481,14 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     uint32_t ph = 0;
     bool ok = true;
     constexpr uint32_t kOperandTx = C::kABytes + C::kBBytes;       // per CTA, signalled on the leader's barrier
+    ACCOUNT_VARS(a_wait = 0, a_total = -ACCOUNT_NOW());
     for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
       int tm, tn;
       tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
       const int m0 = tm * 256 + (int)rank * 128, n0 = tn * BN + (int)rank * (BN / 2);
       for (int ks = 0; ks < p.k_stages; ++ks) {
-        if (!(ok = mbar_wait_relaxed(empty_bar(s), ph ^ 1u, abort_flag, 0x11))) break;
+        ACCOUNT(a_wait, ok = mbar_wait_relaxed(empty_bar(s), ph ^ 1u, abort_flag, 0x11));
+        if (!ok) break;
         const uint32_t st = smem_base + s * C::kStageBytes;
         const uint32_t lead_full = map_to_cta(full_bar(s), 0);
         if (issuer) {
@@ -689,6 +499,8 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         if (++s == C::kStages) { s = 0; ph ^= 1u; }
       }
     }
+    ACCOUNT_STORE(pair == 0 && rank == 0 && issuer, 0, a_wait);
+    ACCOUNT_STORE(pair == 0 && rank == 0 && issuer, 1, a_total + ACCOUNT_NOW());
     if (!ok && issuer) {                            // give copies in flight a bounded time to land
       const unsigned long long t0 = global_timer_ns();
       while (global_timer_ns() - t0 < 200000ull) {}
@@ -734,16 +546,20 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
       int s = 0, b = 0, acc = 0;
       uint32_t ph = 0, bph = 0, acc_ph = 0;
       bool ok = true;
+      ACCOUNT_VARS(a_acc = 0, a_ops = 0, a_sf = 0, a_total = -ACCOUNT_NOW());
       for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
         int tm_unused, tn;
         tile_coords(tile, p.tiles_m, p.tiles_n, tm_unused, tn);
         const uint32_t sfb_off = (uint32_t)((tn * BN) % 128) / 32;         // first scale column of this N tile
-        if (!(ok = mbar_wait_issuer(tempty_bar(acc), acc_ph ^ 1u, abort_flag, 0x12))) break;
+        ACCOUNT(a_acc, ok = mbar_wait_issuer(tempty_bar(acc), acc_ph ^ 1u, abort_flag, 0x12));
+        if (!ok) break;
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int ks = 0; ks < p.k_stages; ++ks) {
-          if (!(ok = mbar_wait_issuer(full_bar(s), ph, abort_flag, 0x13))) break;
+          ACCOUNT(a_ops, ok = mbar_wait_issuer(full_bar(s), ph, abort_flag, 0x13));
+          if (!ok) break;
           if constexpr (!BF16_IN) {
-            if (!(ok = mbar_wait_issuer(sfr_bar(b), bph, abort_flag, 0x15))) break;
+            ACCOUNT(a_sf, ok = mbar_wait_issuer(sfr_bar(b), bph, abort_flag, 0x15));
+            if (!ok) break;
           }
           tc_fence_after();
           const uint32_t st = smem_base + s * C::kStageBytes;
@@ -781,6 +597,10 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         if (issuer) tc_commit_pair(tfull_bar(acc));
         if (++acc == C::kAccStages) { acc = 0; acc_ph ^= 1u; }
       }
+      ACCOUNT_STORE(pair == 0 && issuer, 4, a_acc);
+      ACCOUNT_STORE(pair == 0 && issuer, 5, a_ops);
+      ACCOUNT_STORE(pair == 0 && issuer, 6, a_sf);
+      ACCOUNT_STORE(pair == 0 && issuer, 7, a_total + ACCOUNT_NOW());
     }
   } else if (warp >= 6) {                           // warps 6-9 (warp 10 was taken above)
     // ------------------------------- scale movers (both CTAs) -------------------------------
@@ -792,14 +612,17 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     int s = 0, b = 0;
     uint32_t ph = 0, bph = 0;
     bool ok = true;
+    ACCOUNT_VARS(a_land = 0, a_free = 0, a_total = -ACCOUNT_NOW());
     for (int tile = pair; !BF16_IN && ok && tile < num_tiles; tile += num_pairs) {
       for (int ks = 0; ks < p.k_stages; ++ks) {
-        if (!(ok = mbar_wait_warp_relaxed(sfl_bar(s), ph, abort_flag, 0x16))) break;
+        ACCOUNT(a_land, ok = mbar_wait_warp_relaxed(sfl_bar(s), ph, abort_flag, 0x16));
+        if (!ok) break;
         if constexpr (!C::kSfFollowsStage) {
-          if (!(ok = mbar_wait_warp_relaxed(sfe_bar(b), bph ^ 1u, abort_flag, 0x17))) break;
+          ACCOUNT(a_free, ok = mbar_wait_warp_relaxed(sfe_bar(b), bph ^ 1u, abort_flag, 0x17));
         } else {                                    // buffer b == stage s: free once that stage's previous MMAs are done
-          if (!(ok = mbar_wait_warp_relaxed(empty_bar(s), ph ^ 1u, abort_flag, 0x17))) break;
+          ACCOUNT(a_free, ok = mbar_wait_warp_relaxed(empty_bar(s), ph ^ 1u, abort_flag, 0x17));
         }
+        if (!ok) break;
         tc_fence_after();
         const uint8_t* sf = smem_gen + s * C::kStageBytes + C::kABytes + C::kBBytes + lane * 16;
         const uint32_t t_sf = tmem_base + C::kSfaCol + b * C::kSfCols + lane_field;
@@ -833,6 +656,9 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         if (++b == C::kSfBufs) { b = 0; bph ^= 1u; }
       }
     }
+    ACCOUNT_STORE(pair == 0 && rank == 0 && warp == 6 && lane == 0, 8, a_land);
+    ACCOUNT_STORE(pair == 0 && rank == 0 && warp == 6 && lane == 0, 9, a_free);
+    ACCOUNT_STORE(pair == 0 && rank == 0 && warp == 6 && lane == 0, 10, a_total + ACCOUNT_NOW());
   } else {
     // ------------------------------- epilogue (both CTAs, warps 2-5) -------------------------------
     const int quarter = warp & 3;
@@ -844,10 +670,15 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     int acc = 0;
     uint32_t acc_ph = 0, chunk_no = 0;
     bool ok = true;
+    ACCOUNT_VARS(a_tile = 0, a_read = 0, a_total = -ACCOUNT_NOW(), a_read_t0 = 0);
     for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
       int tm, tn;
-        tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
-      if (!(ok = mbar_wait_warp(tfull_bar(acc), acc_ph, abort_flag, 0x14))) break;
+      tile_coords(tile, p.tiles_m, p.tiles_n, tm, tn);
+      ACCOUNT(a_tile, ok = mbar_wait_warp(tfull_bar(acc), acc_ph, abort_flag, 0x14));
+      if (!ok) break;
+#ifdef NVFP4_GEMM_ACCOUNT
+      a_read_t0 = clock64();
+#endif
       tc_fence_after();
       const int row0 = tm * 256 + (int)rank * 128 + quarter * 32;
       const uint32_t t_row = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
@@ -987,6 +818,9 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(lead_tempty0 + 8u * acc);
+#ifdef NVFP4_GEMM_ACCOUNT
+          a_read += clock64() - a_read_t0;
+#endif
         }
         store_chunk(c * kChunkCols, w);
       }
@@ -995,6 +829,9 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
       if (++acc == C::kAccStages) { acc = 0; acc_ph ^= 1u; }
     }
     if (lane == 0) tma_store_wait_all();
+    ACCOUNT_STORE(pair == 0 && rank == 0 && warp == 2 && lane == 0, 12, a_tile);
+    ACCOUNT_STORE(pair == 0 && rank == 0 && warp == 2 && lane == 0, 13, a_read);
+    ACCOUNT_STORE(pair == 0 && rank == 0 && warp == 2 && lane == 0, 14, a_total + ACCOUNT_NOW());
   }
 
   tc_fence_before();
@@ -1276,3 +1113,15 @@ extern "C" int nvfp4_device_error_word(uint32_t* host_out) {
   *host_out = w;
   return NVFP4_OK;
 }
+
+#ifdef NVFP4_GEMM_ACCOUNT
+// Debug builds only: the cycle account of the last CTA-pair launch (32 values, host pointer).
+//   [0] operand producer: waiting for a free stage   [1] its total
+//   [4] issuer: waiting for the accumulator          [5] waiting for operands   [6] waiting for scales   [7] its total
+//   [8] scale mover: waiting for scale tiles to land [9] waiting for a free scale buffer   [10] its total
+//   [12] epilogue warp: waiting for a finished tile  [13] reading the accumulator out      [14] its total
+extern "C" NVFP4_API int nvfp4_debug_gemm_account(long long* host_out) {
+  if (!host_out) return NVFP4_ERR_NULL;
+  return cudaMemcpyFromSymbol(host_out, g_account, sizeof(long long) * 32) == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+}
+#endif
