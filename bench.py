@@ -4,13 +4,19 @@
 One "step" is one pass of the whole hot path over one Llama-7B-shaped transformer block's five
 linear layers (tokens 16384, hidden 4096): for each layer the forward product (Eq. 1/4), the
 input-gradient product (Eq. 2/5) and the weight-gradient product (Eq. 3/6), each with its
-per-tensor amax passes, its two operand quantizations and its block-scaled GEMM, all through
-the C-ABI entry points nvfp4_linear_fwd / nvfp4_linear_bwd_dx / nvfp4_linear_bwd_dw.
+per-tensor amax passes, its operand quantizations and its block-scaled GEMM, all through the C-ABI
+layer calls nvfp4_linear_fwd_save / nvfp4_linear_bwd_saved.
 
-Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample of
-the same workload instead.
+Prints ONE JSON line (rank 0).  Beside the headline it carries: the GEMM's roofline record (every
+GEMM launch of the workload bracketed by CUDA events, against the measured peaks and against the
+tensor pipe's own issue rate measured in the same run), the quantizer bandwidths, the other
+workload configurations (350M block, 65536-token weight gradient, delayed per-tensor scales, bf16
+outputs, quantization fused into the producing GEMM), the end-to-end figure with host buffers and
+the CPU oracle timed on the host cores.  `--impl reference` times the CPU oracle on a bounded
+sample of the same workload instead.
 """
 import argparse
+import ctypes as C
 import json
 import os
 import statistics
@@ -26,6 +32,8 @@ from paper_2505_19115_b200 import replicas, synth  # noqa: E402
 
 METRIC = "NVFP4 linear fwd+bwd TFLOPS (% FP4 peak); quantizer GB/s (% HBM peak)"
 FP4_OVER_BF16 = 4.0        # nominal dense ratio: 9 PFLOP/s NVFP4 vs 2.25 PFLOP/s bf16
+NOMINAL_FP4_TFLOPS = 9000.0
+MMA_FLOP_PER_CLK_PER_SM = 32768.0   # 2 * 256 * 256 * 64 FLOP per 128 cycles on a CTA pair (microbench mma_peak measures it)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic of the GEMM kernel from the committed ncu capture (profiles/gemm2_nvfp4_kernel_8192x8192x4096.md):
 # 83.0 MB read + 212.2 MB written for 306.2 MB of algorithmic bytes (operand codes and scales + fp32 output).
@@ -50,7 +58,7 @@ def block_flops(cfg):
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
     """Samples SM clock, power and the clock-event reasons of one GPU through NVML from a host
-    thread (every 10 ms) while the timed region runs."""
+    thread (every 10 ms) while a timed region runs."""
     REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20),
                ("sw_power_cap", 0x4))
 
@@ -89,6 +97,7 @@ class ClockSampler:
         import threading
         self.thread = threading.Thread(target=self._run, daemon=True)
         self.thread.start()
+        return self
 
     def mark(self):
         """Drops what was sampled so far (warm-up), so the record covers the timed region only."""
@@ -111,9 +120,9 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
-# reference arm: the CPU oracle on a bounded sample
+# the CPU oracle on the host cores (a reported baseline, not a target)
 # ------------------------------------------------------------------------------------------------
-def oracle_sample_step(cfg, rows=256, seed=2004):
+def oracle_sample_step(cfg, rows=256, seed=2004, nthreads=None):
     """One bounded sample of the workload on the host: the first layer's forward product for the
     first `rows` tokens (quantize those rows of X, quantize all of W, dequantize-then-matmul)."""
     from oracle import binding as ob
@@ -122,13 +131,42 @@ def oracle_sample_step(cfg, rows=256, seed=2004):
     W = synth.normal((N, K), 0.02, seed + 1, device="cpu").float().numpy()
     t0 = time.perf_counter()
     gx, gw = ob.tensor_amax_scale(X), ob.tensor_amax_scale(W)
-    xc, xs = ob.quantize(X, g=gx)
-    wc, ws = ob.quantize(W, g=gw)
-    ob.gemm(xc, xs, gx, wc, ws, gw, want_T=False)
+    xc, xs = ob.quantize(X, g=gx, nthreads=nthreads)
+    wc, ws = ob.quantize(W, g=gw, nthreads=nthreads)
+    ob.gemm(xc, xs, gx, wc, ws, gw, want_T=False, nthreads=nthreads)
     dt = time.perf_counter() - t0
     flops = 2.0 * rows * K * N
     return flops, dt, f"layer '{name}' forward product on the first {rows} of {cfg['tokens']} tokens " \
                       f"(quantize X rows + all of W, dequantize-then-matmul in double)"
+
+
+def cpu_baseline_record(cfg):
+    """The oracle as it stands on the host cores: the forward-product slice at all cores and at one thread
+    (with the linear extrapolation to the whole block step labelled as such) and its quantizer on a whole
+    2^24-element tensor in GB/s at both thread counts.  About 20-30 s of CPU work."""
+    from oracle import binding as ob
+    cores = ob.host_threads()
+    f_all, s_all, sample = oracle_sample_step(cfg, rows=256)
+    f_one, s_one, _ = oracle_sample_step(cfg, rows=16, nthreads=1)
+    tf_all, tf_one = f_all / s_all / 1e12, f_one / s_one / 1e12
+    x = synth.heavy_tailed(synth.square_shape(2 ** 24), seed=1001, device="cpu").float().numpy()
+    g = ob.tensor_amax_scale(x)
+    qbytes = x.size * 2.5625                       # the bf16 source's bytes, as for the GPU figure
+    quant = {"elements": int(x.size), "bytes_per_element": 2.5625}
+    for label, mode in (("rtn", ob.RTN), ("sr", ob.SR)):
+        for tl, nt in (("all_cores", cores), ("1_thread", 1)):
+            t0 = time.perf_counter()
+            ob.quantize(x, g=g, mode=mode, seed=1, nthreads=nt)
+            quant[f"row_{label}_{tl}_GBs"] = qbytes / (time.perf_counter() - t0) / 1e9
+    step_flops = block_flops(cfg)
+    return {"value": tf_all, "unit": "TFLOPS", "cores": cores, "kind": "oracle",
+            "sample": sample + f"; {s_all:.1f} s on {cores} threads",
+            "matmul_slice": {"all_cores_TFLOPS": tf_all, "all_cores_rows": 256, "one_thread_TFLOPS": tf_one,
+                             "one_thread_rows": 16,
+                             "extrapolated_block_step_s_all_cores": step_flops / (tf_all * 1e12),
+                             "extrapolated_block_step_s_one_thread": step_flops / (tf_one * 1e12),
+                             "extrapolation": "linear in FLOPs from the measured slice (labelled estimate, not a measurement)"},
+            "quantizer_2p24": quant}
 
 
 def run_reference(args):
@@ -137,12 +175,13 @@ def run_reference(args):
         return
     from oracle import binding as ob
     cfg = synth.LLAMA_7B
+    rows = 64                                    # about two seconds per step on 16 cores, so that K steps stay within minutes
     for _ in range(max(args.warmup, 0) and 1):
-        oracle_sample_step(cfg)
+        oracle_sample_step(cfg, rows=rows)
     flops = secs = 0.0
     sample = ""
     for _ in range(args.steps):
-        f, dt, sample = oracle_sample_step(cfg)
+        f, dt, sample = oracle_sample_step(cfg, rows=rows)
         flops += f
         secs += dt
     val = flops / secs / 1e12
@@ -162,6 +201,224 @@ def run_reference(args):
 # ------------------------------------------------------------------------------------------------
 # the GPU arm
 # ------------------------------------------------------------------------------------------------
+class Block:
+    """The five linear layers of one transformer block with resident inputs and outputs, and the fused
+    layer calls that make one step: forward (Eq. 1/4) keeping Q(X^T), Q(W^T); backward + update
+    (Eq. 2/5, 3/6) from one read of dY.  Each tensor's amax is taken once, each tensor read once per pass."""
+
+    def __init__(self, nb, cfg, dev, rank, act_dtype=torch.float32, dw_dtype=torch.float32):
+        self.nb, self.cfg, self.M = nb, cfg, cfg["tokens"]
+        M = self.M
+        self.layers = []
+        for li, (name, K, N) in enumerate(cfg["linears"]):
+            X, W, dY = synth.linear_inputs(M, K, N, seed=replicas.replica_seed(4000 + 10 * li, rank), device=dev)
+            self.layers.append(dict(name=name, K=K, N=N, X=X, W=W, dY=dY,
+                                    Y=torch.empty((M, N), dtype=act_dtype, device=dev),
+                                    dX=torch.empty((M, K), dtype=act_dtype, device=dev),
+                                    dW=torch.empty((N, K), dtype=dw_dtype, device=dev)))
+        ws_bytes = max(nb.nvfp4_linear_fused_workspace_bytes(M, l["N"], l["K"], w) for l in self.layers
+                       for w in (nb.FUSED_FWD_SAVE, nb.FUSED_BWD_SAVED))
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        self.saved = torch.empty(max(nb.nvfp4_linear_saved_bytes(M, l["N"], l["K"]) for l in self.layers),
+                                 dtype=torch.uint8, device=dev)
+        self.rt = nb.Rounding(nb.RTN)
+        self.sr = [nb.Rounding(nb.SR, 0, o) for o in range(3)]      # distinct offsets per SR site
+        self.in_bytes = sum(t.numel() * t.element_size() for l in self.layers for t in (l["X"], l["W"], l["dY"]))
+        self.flops = block_flops(cfg)
+        self.given = None
+
+    def compute_given_scales(self):
+        """Per-tensor scales computed once, as a training loop with delayed scaling would carry them over."""
+        nb = self.nb
+        self.given = [{k: nb.nvfp4_tensor_amax_scale(l[k]) for k in ("X", "W", "dY")} for l in self.layers]
+
+    def layer(self, l, gmode, g=None):
+        nb, rt, sr = self.nb, self.rt, self.sr
+        gx, gw, gdy = (g["X"], g["W"], g["dY"]) if g else (None, None, None)
+        nb.nvfp4_linear_fwd_save(l["X"], l["W"], gmode, gx=gx, gw=gw, rx=rt, rw=rt, rxt=sr[2], rwt=rt, out=l["Y"],
+                                 saved=self.saved, workspace=self.ws)
+        nb.nvfp4_linear_bwd_saved(l["dY"], self.saved, l["K"], gmode, gdy=gdy, rdy=sr[0], rdyt=sr[1], dX=l["dX"],
+                                  dW=l["dW"], workspace=self.ws)
+
+    def step(self, gmode=None):
+        gmode = self.nb.G_AMAX if gmode is None else gmode
+        for i, l in enumerate(self.layers):
+            self.layer(l, gmode, self.given[i] if gmode == self.nb.G_GIVEN else None)
+
+    def launches_per_step(self, gmode=None):
+        per_layer = 3 + 3 if gmode == self.nb.G_GIVEN else 3 + 3 + 3   # dual quantizers, GEMMs (+ amax sweeps)
+        return len(self.layers) * per_layer
+
+
+def timed_graph(step, steps, barrier, use_graph=True, sampler=None):
+    """W warm-up steps are the caller's; captures `step` into a CUDA graph (one replay untimed) and times
+    `steps` replays with CUDA events.  Returns (ms_total, launch_mode)."""
+    run, mode = step, "stream"
+    if use_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            graph.replay()
+            run, mode = graph.replay, "cuda_graph"
+        except Exception as e:                  # capture refused: time the plain launches and say so
+            mode = f"stream (graph capture failed: {type(e).__name__})"
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if sampler is not None:
+        sampler.mark()
+    e0.record()
+    for _ in range(steps):
+        run()
+    e1.record()
+    barrier()
+    return e0.elapsed_time(e1), mode
+
+
+def time_call(fn, reps, warm=3, graph=False):
+    """Milliseconds per call (CUDA events).  graph=True replays `reps` calls from one CUDA graph, which keeps the
+    host's launch cost (10-20 us per call from Python) out of the figure for kernels that run only a few microseconds."""
+    for _ in range(warm):
+        fn()
+    run, n = fn, reps
+    if graph:
+        try:
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for _ in range(reps):
+                    fn()
+            g.replay()
+            run, n = g.replay, 1
+        except Exception:
+            run, n = fn, reps
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def quantizer_sweep(nb, dev, peaks, peak_kind):
+    """Quantizer bandwidth on the heavy-tailed tensors: 2^28 elements (exceeds L2: the HBM figure) and, labelled
+    as L2-resident and launch-bound, 2^24 and 2^20.  Bytes = 2 + 0.5 + 1/16 per element (3.125 for both orientations)."""
+    rt = nb.Rounding(nb.RTN)
+    out = {"bytes_per_element": 2.5625, "peak_hbm_gbs": peaks["hbm_gbs"], "peak_kind": peak_kind}
+    L = nb.lib()
+    for n_el, reps, note in ((2 ** 28, 10, None),
+                             (2 ** 24, 30, "L2-resident: 32 MiB of input, not an HBM figure; back-to-back launches replayed from a CUDA graph"),
+                             (2 ** 20, 50, "L2-resident and launch-bound: 2 MiB of input, a few microseconds per launch; back-to-back "
+                                           "launches replayed from a CUDA graph")):
+        small = n_el < 2 ** 28
+        xq = synth.heavy_tailed(synth.square_shape(n_el), seed=1002, device=dev)
+        R, Cc = xq.shape
+        gq = nb.nvfp4_tensor_amax_scale(xq)
+        codes = torch.empty((R, Cc // 2), dtype=torch.uint8, device=dev)
+        sfs = torch.empty(nb.nvfp4_sf_bytes(R, Cc, nb.SF_SWIZZLED), dtype=torch.uint8, device=dev)
+        ct = torch.empty((Cc, R // 2), dtype=torch.uint8, device=dev)
+        st = torch.empty(nb.nvfp4_sf_bytes(Cc, R, nb.SF_SWIZZLED), dtype=torch.uint8, device=dev)
+        rec = {"elements": n_el}
+        if note:
+            rec["note"] = note
+        for label, tr, rr in (("row_rtn", False, rt), ("row_sr", False, nb.Rounding(nb.SR, 1, 0)),
+                              ("transposed_rtn", True, rt), ("transposed_sr", True, nb.Rounding(nb.SR, 1, 0))):
+            c_, s_ = (ct, st) if tr else (codes, sfs)
+            ms = time_call(lambda: nb.nvfp4_quantize(xq, tr, gq, rr, nb.SF_SWIZZLED, codes=c_, scales=s_), reps, graph=small)
+            gbs = n_el * 2.5625 / (ms * 1e-3) / 1e9
+            rec[label] = {"GB/s": gbs, "us": ms * 1e3, "frac_of_measured_copy": gbs / peaks["hbm_gbs"], "frac_of_8TBs": gbs / 8000.0}
+        # both orientations from one read (the fused layer's quantizer): 2 + 2 * 0.5625 bytes per element
+        for label, r1, r2 in (("dual_rtn", rt, rt), ("dual_sr", nb.Rounding(nb.SR, 1, 0), nb.Rounding(nb.SR, 1, 1))):
+            def dual():
+                stt = L.nvfp4_quantize_dual(xq.data_ptr(), nb.BF16, R, Cc, xq.stride(0), gq.data_ptr(),
+                                            C.byref(r1), codes.data_ptr(), sfs.data_ptr(), C.byref(r2), ct.data_ptr(),
+                                            st.data_ptr(), nb.SF_SWIZZLED, torch.cuda.current_stream().cuda_stream)
+                assert stt == 0
+            ms = time_call(dual, reps, graph=small)
+            gbs = n_el * 3.125 / (ms * 1e-3) / 1e9
+            rec[label] = {"GB/s": gbs, "us": ms * 1e3, "bytes_per_element": 3.125,
+                          "frac_of_measured_copy": gbs / peaks["hbm_gbs"], "frac_of_8TBs": gbs / 8000.0}
+        ms = time_call(lambda: nb.nvfp4_tensor_amax_scale(xq, out=gq), reps, graph=small)
+        rec["amax"] = {"GB/s": n_el * 2.0 / (ms * 1e-3) / 1e9, "us": ms * 1e3, "bytes_per_element": 2.0}
+        if n_el == 2 ** 28:
+            out.update(rec)                     # the HBM figures stay at the top level of the record
+        else:
+            out[f"elements_2p{n_el.bit_length() - 1}"] = rec
+        del xq, codes, sfs, ct, st
+        torch.cuda.empty_cache()
+    return out
+
+
+def long_token_axis_leg(nb, dev):
+    """The FFN weight-gradient product with a 65536-token contraction (Eq. 3/6): dW = dY^T X, dY 65536 x 11008,
+    X 65536 x 4096, both SR-quantized in blocks along the tokens."""
+    t = synth.LONG_DW
+    M, K, N = t["tokens"], t["K"], t["N"]
+    dY = synth.normal((M, N), 1e-4, 2005, device=dev)
+    X = synth.normal((M, K), 1.0, 2006, device=dev)
+    r_dy, r_x = nb.Rounding(nb.SR, 2, 1), nb.Rounding(nb.SR, 2, 2)
+    dW = torch.empty((N, K), dtype=torch.float32, device=dev)
+    ws = torch.empty(nb.nvfp4_linear_workspace_bytes(M, N, K, nb.LINEAR_BWD_DW), dtype=torch.uint8, device=dev)
+    flops = 2.0 * M * N * K
+    ms_e2e = time_call(lambda: nb.nvfp4_linear_bwd_dw(dY, X, nb.G_AMAX, rdy=r_dy, rx=r_x, out=dW, workspace=ws), 5, warm=2)
+    gdy, gx = nb.nvfp4_tensor_amax_scale(dY), nb.nvfp4_tensor_amax_scale(X)
+    ac, asf = nb.nvfp4_quantize(dY, True, gdy, r_dy, nb.SF_SWIZZLED)
+    bc, bsf = nb.nvfp4_quantize(X, True, gx, r_x, nb.SF_SWIZZLED)
+    ms_q = [time_call(lambda: nb.nvfp4_quantize(dY, True, gdy, r_dy, nb.SF_SWIZZLED, codes=ac, scales=asf), 5, warm=2),
+            time_call(lambda: nb.nvfp4_quantize(X, True, gx, r_x, nb.SF_SWIZZLED, codes=bc, scales=bsf), 5, warm=2)]
+    ms_gemm = time_call(lambda: nb.nvfp4_gemm(ac, asf, gdy, bc, bsf, gx, out=dW), 10, warm=2)
+    return {"workload": "ffn_weight_gradient_65536_tokens", "M_tokens": M, "N": N, "K": K, "flops": flops,
+            "gemm_only_TFLOPS": flops / ms_gemm / 1e9, "gemm_ms": ms_gemm,
+            "end_to_end_TFLOPS": flops / ms_e2e / 1e9, "end_to_end_ms": ms_e2e,
+            "end_to_end_is": "amax x2 + transposed SR quantizers x2 + GEMM, through nvfp4_linear_bwd_dw",
+            "transposed_sr_quantizer_GBs": {"dY": M * N * 2.5625 / ms_q[0] / 1e6, "X": M * K * 2.5625 / ms_q[1] / 1e6}}
+
+
+def fused_producer_leg(nb, dev, cfg):
+    """Quantization fused into the producing GEMM (no bf16/fp32 round trip): the up projection's product leaves
+    its GEMM already quantized along its feature axis and feeds the down projection (the position of the SwiGLU
+    output in Section 5's model; the activation itself is not part of this library).  Against the unfused pair:
+    fp32 product, then nvfp4_quantize."""
+    M = cfg["tokens"]
+    (_, K1, N1), (_, K2, N2) = [l for l in cfg["linears"] if l[0] in ("up", "down")]
+    assert N1 == K2
+    X, W1, _ = synth.linear_inputs(M, K1, N1, seed=4100, device=dev)
+    _, W2, _ = synth.linear_inputs(M, K2, N2, seed=4101, device=dev)
+    rt = nb.Rounding(nb.RTN)
+    gx, g1, g2 = nb.nvfp4_tensor_amax_scale(X), nb.nvfp4_tensor_amax_scale(W1), nb.nvfp4_tensor_amax_scale(W2)
+    xc, xs = nb.nvfp4_quantize(X, False, gx, rt, nb.SF_SWIZZLED)
+    w1c, w1s = nb.nvfp4_quantize(W1, False, g1, rt, nb.SF_SWIZZLED)
+    w2c, w2s = nb.nvfp4_quantize(W2, False, g2, rt, nb.SF_SWIZZLED)
+    H = torch.empty((M, N1), dtype=torch.float32, device=dev)
+    Y = torch.empty((M, N2), dtype=torch.float32, device=dev)
+    nb.nvfp4_gemm(xc, xs, gx, w1c, w1s, g1, out=H)
+    gh = nb.nvfp4_tensor_amax_scale(H)              # the consumer's per-tensor scale must be known beforehand (delayed scaling)
+    hc = torch.empty((M, N1 // 2), dtype=torch.uint8, device=dev)
+    hs = torch.empty(nb.nvfp4_sf_bytes(M, N1, nb.SF_SWIZZLED), dtype=torch.uint8, device=dev)
+    L = nb.lib()
+
+    def fused():
+        st = L.nvfp4_gemm_quantized(xc.data_ptr(), xs.data_ptr(), gx.data_ptr(), w1c.data_ptr(), w1s.data_ptr(), g1.data_ptr(),
+                                    M, N1, K1, gh.data_ptr(), C.byref(rt), hc.data_ptr(), hs.data_ptr(), nb.SF_SWIZZLED,
+                                    torch.cuda.current_stream().cuda_stream)
+        assert st == 0
+        nb.nvfp4_gemm(hc, hs, gh, w2c, w2s, g2, out=Y)
+
+    def unfused():
+        nb.nvfp4_gemm(xc, xs, gx, w1c, w1s, g1, out=H)
+        nb.nvfp4_quantize(H, False, gh, rt, nb.SF_SWIZZLED, codes=hc, scales=hs)
+        nb.nvfp4_gemm(hc, hs, gh, w2c, w2s, g2, out=Y)
+
+    ms_f, ms_u = time_call(fused, 10), time_call(unfused, 10)
+    flops = 2.0 * M * (K1 * N1 + K2 * N2)
+    return {"workload": "up projection -> quantized in its epilogue -> down projection", "M": M, "K1": K1, "N1": N1, "N2": N2,
+            "fused_ms": ms_f, "unfused_ms": ms_u, "time_saved_ms": ms_u - ms_f,
+            "fused_TFLOPS": flops / ms_f / 1e9, "unfused_TFLOPS": flops / ms_u / 1e9,
+            "bytes_not_moved": M * N1 * 8,         # the fp32 intermediate is neither written nor read back
+            "bytes_note": "the M x N1 fp32 intermediate: 4 B/element written by the first GEMM + 4 B/element read by the quantizer"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -172,6 +429,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-quantizer", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the legs for the other workload configurations")
     ap.add_argument("--no-graph", action="store_true", help="launch every step kernel by kernel instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -180,6 +438,7 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     from paper_2505_19115_b200 import binding as nb
+    from paper_2505_19115_b200 import microbench
 
     rank, world, local = replicas.env_rank_world()
     torch.cuda.set_device(local)
@@ -192,39 +451,8 @@ def main():
     nb.lib()                                      # fails loudly when the CUDA library is missing
 
     cfg = synth.LLAMA_7B if args.workload == "llama7b" else synth.LLAMA_350M
-    M = cfg["tokens"]
     peaks, peak_kind = load_peaks()
-
-    # ---- resident inputs: every rank has its own block (replicas; no data-path collective) ----
-    layers = []
-    for li, (name, K, N) in enumerate(cfg["linears"]):
-        X, W, dY = synth.linear_inputs(M, K, N, seed=replicas.replica_seed(4000 + 10 * li, rank), device=dev)
-        layers.append(dict(name=name, K=K, N=N, X=X, W=W, dY=dY,
-                           Y=torch.empty((M, N), dtype=torch.float32, device=dev),
-                           dX=torch.empty((M, K), dtype=torch.float32, device=dev),
-                           dW=torch.empty((N, K), dtype=torch.float32, device=dev)))
-    ws_bytes = max(nb.nvfp4_linear_fused_workspace_bytes(M, l["N"], l["K"], w) for l in layers
-                   for w in (nb.FUSED_FWD_SAVE, nb.FUSED_BWD_SAVED))
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
-    saved = torch.empty(max(nb.nvfp4_linear_saved_bytes(M, l["N"], l["K"]) for l in layers), dtype=torch.uint8, device=dev)
-    rt = nb.Rounding(nb.RTN)
-    sr = [nb.Rounding(nb.SR, 0, o) for o in range(3)]      # distinct offsets per SR site
-    in_bytes = sum(t.numel() * t.element_size() for l in layers for t in (l["X"], l["W"], l["dY"]))
-
-    def layer_fwd_bwd(l):
-        # forward (Eq. 1/4) keeping Q(X^T), Q(W^T); backward + update (Eq. 2/5, 3/6) from one read of dY.
-        # Each tensor's amax is taken once, each tensor is read once per pass.
-        nb.nvfp4_linear_fwd_save(l["X"], l["W"], nb.G_AMAX, rx=rt, rw=rt, rxt=sr[2], rwt=rt, out=l["Y"], saved=saved,
-                                 workspace=ws)
-        nb.nvfp4_linear_bwd_saved(l["dY"], saved, l["K"], nb.G_AMAX, rdy=sr[0], rdyt=sr[1], dX=l["dX"], dW=l["dW"],
-                                  workspace=ws)
-
-    def step():
-        for l in layers:
-            layer_fwd_bwd(l)
-
-    launches_per_step = len(layers) * (3 + 3 + 3)         # 3 amax sweeps, 3 dual quantizers, 3 GEMMs per layer
-    flops_per_step = block_flops(cfg)
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
 
     def barrier():
         torch.cuda.synchronize()
@@ -232,59 +460,40 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
+    # ---- the headline: resident inputs, every rank its own block (replicas; no data-path collective) ----
+    block = Block(nb, cfg, dev, rank)
+    M = block.M
+    layers = block.layers
+    sampler = ClockSampler(local).start() if rank == 0 else None
     for _ in range(args.warmup):
-        step()
+        block.step()
     barrier()
-    # One step = 60 launches of 20-400 us: captured once into a CUDA graph (after the warm-up, so that every
+    # One step = 45 launches of 20-400 us: captured once into a CUDA graph (after the warm-up, so that every
     # one-time set-up inside the library is done) and replayed, which removes the launch gaps between them.
-    # The graph holds exactly the calls of step(), on the same buffers.
-    run_step, launch_mode = step, "stream"
-    if not args.no_graph:
-        try:
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph):
-                step()
-            graph.replay()                      # one more untimed step, through the graph
-            run_step, launch_mode = graph.replay, "cuda_graph"
-        except Exception as e:                  # capture refused: time the plain launches and say so
-            launch_mode = f"stream (graph capture failed: {type(e).__name__})"
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    sampler.mark()
-    e0.record()
-    for _ in range(args.steps):
-        run_step()
-    e1.record()
-    barrier()
+    ms, launch_mode = timed_graph(block.step, args.steps, barrier, not args.no_graph, sampler)
     clocks = sampler.stop() if rank == 0 else None
-    ms = e0.elapsed_time(e1)
     ms = replicas.max_over_ranks(ms, dist, dev)
     err_word = nb.nvfp4_device_error_word()
     if err_word:
         raise RuntimeError(f"device error word {err_word:#x}: a kernel gave up on a bounded wait")
+    flops_per_step = block.flops
     value = replicas.aggregate_throughput(flops_per_step * args.steps, world, ms * 1e-3) / 1e12
+    launches_per_step = block.launches_per_step()
 
     # ---- roofline of the dominant kernel (the GEMM): same workload, decomposed into the C-ABI's
-    #      quantize and gemm calls so that CUDA events bracket every GEMM launch ----
-    def decomposed_ops(l):
-        ops = []
-        for kind, a, b, ta, tb, ra, rb, out in (("fwd", l["X"], l["W"], False, False, rt, rt, l["Y"]),
-                                                 ("dx", l["dY"], l["W"], False, True, sr[0], rt, l["dX"]),
-                                                 ("dw", l["dY"], l["X"], True, True, sr[1], sr[2], l["dW"])):
-            ops.append((a, b, ta, tb, ra, rb, out))
-        return ops
-
-    gemm_events = []
-    gemm_flops = 0.0
-    gemm_bytes = 0.0
-    roof_steps = min(args.steps, 3)
+    #      quantize and gemm calls so that CUDA events bracket every GEMM launch; clocks sampled meanwhile ----
+    rt, sr = block.rt, block.sr
+    roof_sampler = ClockSampler(local).start() if rank == 0 else None
+    gemm_events, gemm_flops, gemm_bytes = [], 0.0, 0.0
+    roof_steps = min(args.steps, 6)
     for it in range(roof_steps + 1):
+        if it == 1 and roof_sampler is not None:
+            torch.cuda.synchronize()
+            roof_sampler.mark()                  # the first pass is warm-up
         for l in layers:
-            for a, b, ta, tb, ra, rb, out in decomposed_ops(l):
+            for a, b, ta, tb, ra, rb, out in ((l["X"], l["W"], False, False, rt, rt, l["Y"]),
+                                               (l["dY"], l["W"], False, True, sr[0], rt, l["dX"]),
+                                               (l["dY"], l["X"], True, True, sr[1], sr[2], l["dW"])):
                 ga, gb = nb.nvfp4_tensor_amax_scale(a), nb.nvfp4_tensor_amax_scale(b)
                 ac, asf = nb.nvfp4_quantize(a, ta, ga, ra, nb.SF_SWIZZLED)
                 bc, bsf = nb.nvfp4_quantize(b, tb, gb, rb, nb.SF_SWIZZLED)
@@ -292,86 +501,119 @@ def main():
                 s0.record()
                 nb.nvfp4_gemm(ac, asf, ga, bc, bsf, gb, out=out)
                 s1.record()
-                if it > 0:                       # first pass is warm-up
+                if it > 0:
                     gemm_events.append((s0, s1))
                     gemm_flops += 2.0 * out.shape[0] * out.shape[1] * ac.shape[1] * 2
                     gemm_bytes += (ac.numel() + bc.numel()) * 1.125 + out.numel() * out.element_size()
                 del ac, asf, bc, bsf
     torch.cuda.synchronize()
+    roof_clocks = roof_sampler.stop() if rank == 0 else None
     gemm_ms = sum(a.elapsed_time(b) for a, b in gemm_events)
     n_gemm = len(gemm_events)
     gemm_tflops = gemm_flops / (gemm_ms * 1e-3) / 1e12
-    fp4_peak = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
+    # The denominator follows from the run: each GEMM launch is timed alone, which is the burst regime while the
+    # clock sampled during this pass stays within 10 % of its maximum; a run that the power cap has pulled below
+    # that is measured against the sustained figure.
+    roof_mhz = (roof_clocks or {}).get("sm_mhz")
+    roof_max = (roof_clocks or {}).get("sm_max_mhz") or peaks.get("sm_max_mhz")
+    burst = not (roof_mhz and roof_max) or roof_mhz >= 0.9 * roof_max
+    bf16_peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
+    fp4_peak = bf16_peak * FP4_OVER_BF16
+    fp4_sustained = peaks["bf16_tflops_sustained"] * FP4_OVER_BF16
+    # the tensor pipe's own ceiling, measured now: the GEMM's instruction issued back to back on resident operands
+    mma = microbench.mma_peak(stages=1024, iters=3, warmup=1) if rank == 0 else None
+    issue_peak_at_clock = sms * MMA_FLOP_PER_CLK_PER_SM * roof_mhz * 1e6 / 1e12 if roof_mhz else None
     roofline = {
         "bound": "tensor", "kernel": "gemm2_nvfp4_kernel<256>", "achieved": gemm_tflops, "peak": fp4_peak, "unit": "TFLOP/s",
         "frac": gemm_tflops / fp4_peak, "traffic": GEMM_TRAFFIC_RATIO * gemm_bytes / n_gemm,
         "traffic_basis": "ncu capture of an 8192x8192x4096 launch (0.96 of its algorithmic bytes), scaled by the "
                          "algorithmic bytes per launch of this workload",
         "algorithmic_bytes_per_launch_avg": gemm_bytes / n_gemm,
-        "peak_basis": f"{peak_kind} sustained bf16 {peaks['bf16_tflops_sustained']} TFLOP/s x {FP4_OVER_BF16:g} "
-                      f"(nominal dense NVFP4/bf16 ratio); burst basis {peaks['bf16_tflops'] * FP4_OVER_BF16:.0f}; nominal 9000",
+        "peak_basis": f"{peak_kind} {'burst' if burst else 'sustained'} bf16 {bf16_peak} TFLOP/s x {FP4_OVER_BF16:g} (nominal dense "
+                      f"NVFP4/bf16 ratio): every GEMM launch is timed alone and the SM clock sampled during this pass had a "
+                      f"median of {roof_mhz} MHz of {roof_max} ({'within' if burst else 'more than'} 10 % of the maximum)",
         "launches": n_gemm, "avg_launch_ms": gemm_ms / n_gemm, "flops_per_launch_avg": gemm_flops / n_gemm,
-        "frac_of_nominal_9pf": gemm_tflops / 9000.0,
+        "frac_of_burst_x4": gemm_tflops / (peaks["bf16_tflops"] * FP4_OVER_BF16),
+        "frac_of_sustained_x4": gemm_tflops / fp4_sustained,
+        "frac_of_nominal_9pf": gemm_tflops / NOMINAL_FP4_TFLOPS,
+        "issue_peak_at_sampled_clock": issue_peak_at_clock,
+        "frac_of_issue_peak": gemm_tflops / issue_peak_at_clock if issue_peak_at_clock else None,
+        "issue_peak_basis": f"{sms} SMs x {MMA_FLOP_PER_CLK_PER_SM:g} FLOP/clk x the sampled median clock",
+        "mma_peak_measured": mma,
+        "frac_of_mma_peak_measured": gemm_tflops / mma["TFLOP/s"] if mma else None,
+        "mma_peak_note": "tcgen05.mma kind::mxf4nvf4 (256x256x64, CTA pair) issued back to back on resident operands in this "
+                         "run: the rate the tensor pipe delivers at the clock it holds under that load (implied_sm_mhz)",
+        "clocks": roof_clocks,
     }
 
-    # ---- quantizer bandwidth at 2^28 elements (heavy-tailed inputs), bytes = 2 + 0.5 + 1/16 per element ----
+    # ---- quantizer bandwidths ----
     quant = None
     if not args.no_quantizer and rank == 0:
         for l in layers:
             l["Y"] = l["dX"] = l["dW"] = None
         torch.cuda.empty_cache()
-        n_el = 2 ** 28
-        xq = synth.heavy_tailed(synth.square_shape(n_el), seed=1002, device=dev)
-        gq = nb.nvfp4_tensor_amax_scale(xq)
-        codes = torch.empty((xq.shape[0], xq.shape[1] // 2), dtype=torch.uint8, device=dev)
-        sfs = torch.empty(nb.nvfp4_sf_bytes(xq.shape[0], xq.shape[1], nb.SF_SWIZZLED), dtype=torch.uint8, device=dev)
-        quant = {"elements": n_el, "bytes_per_element": 2.5625, "peak_hbm_gbs": peaks["hbm_gbs"], "peak_kind": peak_kind}
-        for label, tr, rr in (("row_rtn", False, rt), ("row_sr", False, nb.Rounding(nb.SR, 1, 0)),
-                              ("transposed_rtn", True, rt), ("transposed_sr", True, nb.Rounding(nb.SR, 1, 0))):
-            for _ in range(3):
-                nb.nvfp4_quantize(xq, tr, gq, rr, nb.SF_SWIZZLED, codes=codes, scales=sfs)
-            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            reps = 10
-            q0.record()
-            for _ in range(reps):
-                nb.nvfp4_quantize(xq, tr, gq, rr, nb.SF_SWIZZLED, codes=codes, scales=sfs)
-            q1.record()
-            torch.cuda.synchronize()
-            gbs = n_el * 2.5625 * reps / (q0.elapsed_time(q1) * 1e-3) / 1e9
-            quant[label] = {"GB/s": gbs, "frac_of_measured_copy": gbs / peaks["hbm_gbs"], "frac_of_8TBs": gbs / 8000.0}
-        # both orientations from one read (the fused layer's quantizer): 2 + 2 * 0.5625 bytes per element
-        L = nb.lib()
-        import ctypes as C
-        ct = torch.empty((xq.shape[1], xq.shape[0] // 2), dtype=torch.uint8, device=dev)
-        st = torch.empty(nb.nvfp4_sf_bytes(xq.shape[1], xq.shape[0], nb.SF_SWIZZLED), dtype=torch.uint8, device=dev)
-        for label, r1, r2 in (("dual_rtn", rt, rt), ("dual_sr", nb.Rounding(nb.SR, 1, 0), nb.Rounding(nb.SR, 1, 1))):
-            def dual():
-                stt = L.nvfp4_quantize_dual(xq.data_ptr(), nb.BF16, xq.shape[0], xq.shape[1], xq.stride(0), gq.data_ptr(),
-                                            C.byref(r1), codes.data_ptr(), sfs.data_ptr(), C.byref(r2), ct.data_ptr(),
-                                            st.data_ptr(), nb.SF_SWIZZLED, torch.cuda.current_stream().cuda_stream)
-                assert stt == 0
-            for _ in range(3):
-                dual()
-            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            q0.record()
-            for _ in range(10):
-                dual()
-            q1.record()
-            torch.cuda.synchronize()
-            gbs = n_el * 3.125 * 10 / (q0.elapsed_time(q1) * 1e-3) / 1e9
-            quant[label] = {"GB/s": gbs, "bytes_per_element": 3.125, "frac_of_measured_copy": gbs / peaks["hbm_gbs"],
-                            "frac_of_8TBs": gbs / 8000.0}
-        del xq, codes, sfs, ct, st
+        quant = quantizer_sweep(nb, dev, peaks, peak_kind)
+    for l in layers:
+        for k in ("Y", "dX", "dW"):
+            if l[k] is None:
+                shape = {"Y": (M, l["N"]), "dX": (M, l["K"]), "dW": (l["N"], l["K"])}[k]
+                l[k] = torch.empty(shape, dtype=torch.float32, device=dev)
+
+    # ---- the other workload configurations and modes (single GPU, rank 0; a few seconds in total) ----
+    configs = None
+    if not args.no_configs and rank == 0 and world == 1:
+        configs = {}
+        n_extra = 10
+        # delayed per-tensor scales: the same step with g supplied (no amax sweep inside the timed region)
+        block.compute_given_scales()
+        for _ in range(2):
+            block.step(nb.G_GIVEN)
+        ms_g, _ = timed_graph(lambda: block.step(nb.G_GIVEN), n_extra, barrier, not args.no_graph)
+        configs["step_with_given_scales"] = {
+            "workload": "the headline block step with NVFP4_G_GIVEN: per-tensor scales carried over (delayed scaling), no amax pass",
+            "ms_per_step": ms_g / n_extra, "TFLOPS": flops_per_step * n_extra / ms_g / 1e9,
+            "gpu_launches_per_step": block.launches_per_step(nb.G_GIVEN)}
+        # bf16 activations out (Y, dX), fp32 weight gradient
+        del block.layers[:]
+        del block, layers
         torch.cuda.empty_cache()
+        blk16 = Block(nb, cfg, dev, rank, act_dtype=torch.bfloat16)
+        for _ in range(2):
+            blk16.step()
+        ms_b, _ = timed_graph(blk16.step, n_extra, barrier, not args.no_graph)
+        configs["step_with_bf16_activations"] = {
+            "workload": "the headline block step with bf16 Y and dX and fp32 dW (amax inside the calls)",
+            "ms_per_step": ms_b / n_extra, "TFLOPS": flops_per_step * n_extra / ms_b / 1e9}
+        del blk16.layers[:]
+        del blk16
+        torch.cuda.empty_cache()
+        # the 350M-class block (or the 7B one when that is not the headline)
+        other = synth.LLAMA_350M if args.workload == "llama7b" else synth.LLAMA_7B
+        blk_o = Block(nb, other, dev, rank)
+        for _ in range(3):
+            blk_o.step()
+        n_o = 20
+        ms_o, _ = timed_graph(blk_o.step, n_o, barrier, not args.no_graph)
+        configs["other_block"] = {
+            "workload": ("llama350m" if args.workload == "llama7b" else "llama7b") + "_block_linears_fwd_bwd",
+            "tokens": other["tokens"], "hidden": other["hidden"], "ms_per_step": ms_o / n_o,
+            "TFLOPS": blk_o.flops * n_o / ms_o / 1e9, "flops_per_step": blk_o.flops}
+        del blk_o.layers[:]
+        del blk_o
+        torch.cuda.empty_cache()
+        configs["long_token_axis_weight_gradient"] = long_token_axis_leg(nb, dev)
+        torch.cuda.empty_cache()
+        configs["quantization_fused_into_producer"] = fused_producer_leg(nb, dev, synth.LLAMA_7B)
+        torch.cuda.empty_cache()
+        err_word = nb.nvfp4_device_error_word()
+        if err_word:
+            raise RuntimeError(f"device error word {err_word:#x} in the configuration legs")
+        block = Block(nb, cfg, dev, rank)          # back to the headline block for the end-to-end leg
+        layers = block.layers
 
     # ---- end to end through the C ABI with host buffers (H2D of every input, D2H of every output) ----
     e2e = None
     if not args.no_e2e:
-        for l in layers:
-            for k in ("Y", "dX", "dW"):
-                if l[k] is None:
-                    shape = {"Y": (M, l["N"]), "dX": (M, l["K"]), "dW": (l["N"], l["K"])}[k]
-                    l[k] = torch.empty(shape, dtype=torch.float32, device=dev)
         host_in = [{k: l[k].cpu().pin_memory() for k in ("X", "W", "dY")} for l in layers]
         max_out = {k: max(l[k].numel() for l in layers) for k in ("Y", "dX", "dW")}
         host_out = {k: torch.empty(n, dtype=torch.float32).pin_memory() for k, n in max_out.items()}
@@ -400,7 +642,7 @@ def main():
                     s_cmp.wait_event(ev_in[i])
                     if not first[0]:
                         s_cmp.wait_event(ev_out[i])
-                    layer_fwd_bwd(l)
+                    block.layer(l, nb.G_AMAX)
                     ev_done[i].record(s_cmp)
                 with torch.cuda.stream(s_out):
                     s_out.wait_event(ev_done[i])
@@ -436,23 +678,19 @@ def main():
                "ms_per_step": ems / e2e_steps}
         del host_in, host_out
 
-    # ---- the oracle on the host cores, bounded sample ----
+    # ---- the oracle on the host cores, bounded samples, after every timed GPU region ----
     cpu = None
     if rank == 0 and not args.no_cpu and world == 1:
-        from oracle import binding as ob
-        f = secs = 0.0
-        sample = ""
-        for _ in range(2):
-            ff, dt, sample = oracle_sample_step(cfg)
-            f += ff
-            secs += dt
-        cpu = {"value": f / secs / 1e12, "unit": "TFLOPS", "cores": ob.host_threads(), "kind": "oracle",
-               "sample": sample + f"; 2 repetitions, {secs:.1f} s"}
+        cpu = cpu_baseline_record(cfg)
 
     if rank == 0:
+        ms_step = ms / args.steps
+        mhz = (clocks or {}).get("sm_mhz")
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "warmup": args.warmup, "ms_per_step": ms_step,
+            "ms_x_mhz_per_step": ms_step * mhz if mhz else None,      # separates the power-capped regime from the burst one
+            "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "nvfp4 (e2m1 x ue4m3 block scales), fp32 accumulate and output",
             "data": "synthetic",
             "config": {"workload": "llama7b_block_linears_fwd_bwd" if args.workload == "llama7b" else "llama350m_block_linears_fwd_bwd",
@@ -461,11 +699,13 @@ def main():
                        "per_tensor_scale": "amax/(6*448), computed once per tensor inside the calls",
                        "launch": launch_mode,
                        "fusion": "nvfp4_linear_fwd_save + nvfp4_linear_bwd_saved: X, W, dY each read once per pass, both orientations quantized from that read",
-                       "l2": f"inputs exceed L2: {in_bytes / 2 ** 20:.0f} MiB of operands per step, fp32 outputs on top",
+                       "l2": f"inputs exceed L2: {sum(2 * M * (k + o) + 2 * k * o for _, k, o in cfg['linears']) / 2 ** 20:.0f} MiB of operands per step, fp32 outputs on top",
+                       "timed_region_s": ms * 1e-3,
                        "parallelism": "replicas only (one GPU per rank, no data-path collective)"},
-            "pct_of_fp4_peak": {"of_nominal_9pf": value / world / 9000.0 * 100,
-                                f"of_{peak_kind}_sustained_x4": value / world / fp4_peak * 100},
-            "roofline": roofline, "quantizer": quant, "cpu_baseline": cpu, "e2e": e2e,
+            "pct_of_fp4_peak": {"of_nominal_9pf": value / world / NOMINAL_FP4_TFLOPS * 100,
+                                f"of_{peak_kind}_sustained_x4": value / world / fp4_sustained * 100,
+                                f"of_{peak_kind}_burst_x4": value / world / (peaks["bf16_tflops"] * FP4_OVER_BF16) * 100},
+            "roofline": roofline, "quantizer": quant, "configs": configs, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
         }
         print(json.dumps(line))
