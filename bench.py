@@ -58,12 +58,13 @@ def block_flops(cfg):
 # ------------------------------------------------------------------------------------------------
 class ClockSampler:
     """Samples SM clock, power and the clock-event reasons of one GPU through NVML from a host
-    thread (every 10 ms) while a timed region runs."""
+    thread (every 10 ms unless told otherwise) while a timed region runs."""
     REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20),
                ("sw_power_cap", 0x4))
 
-    def __init__(self, device_index):
+    def __init__(self, device_index, interval_s=0.01):
         self.idx = device_index
+        self.interval_s = interval_s
         self.thread = None
         self.stop_flag = False
         self.sm, self.power, self.mask = [], [], 0
@@ -89,7 +90,7 @@ class ClockSampler:
                     self.mask |= int(pynvml.nvmlDeviceGetCurrentClocksEventReasons(h))
                 except Exception:
                     pass
-                time.sleep(0.01)
+                time.sleep(self.interval_s)
         except Exception as e:  # the number is still reported, without a clock record
             self.error = repr(e)
 
@@ -377,9 +378,10 @@ def long_token_axis_leg(nb, dev):
 
 def fused_producer_leg(nb, dev, cfg):
     """Quantization fused into the producing GEMM (no bf16/fp32 round trip): the up projection's product leaves
-    its GEMM already quantized along its feature axis and feeds the down projection (the position of the SwiGLU
-    output in Section 5's model; the activation itself is not part of this library).  Against the unfused pair:
-    fp32 product, then nvfp4_quantize."""
+    its GEMM already quantized along its feature axis (nvfp4_linear_fwd_qout) and feeds the down projection
+    (nvfp4_linear_fwd_qin) -- the position of the SwiGLU output in Section 5's model; the activation itself is not
+    part of this library.  Against the unfused pair of nvfp4_linear_fwd calls: fp32 intermediate written, read
+    back for its amax and read again by the next layer's quantizer.  Per-tensor scales are given in both arms."""
     M = cfg["tokens"]
     (_, K1, N1), (_, K2, N2) = [l for l in cfg["linears"] if l[0] in ("up", "down")]
     assert N1 == K2
@@ -387,36 +389,43 @@ def fused_producer_leg(nb, dev, cfg):
     _, W2, _ = synth.linear_inputs(M, K2, N2, seed=4101, device=dev)
     rt = nb.Rounding(nb.RTN)
     gx, g1, g2 = nb.nvfp4_tensor_amax_scale(X), nb.nvfp4_tensor_amax_scale(W1), nb.nvfp4_tensor_amax_scale(W2)
-    xc, xs = nb.nvfp4_quantize(X, False, gx, rt, nb.SF_SWIZZLED)
-    w1c, w1s = nb.nvfp4_quantize(W1, False, g1, rt, nb.SF_SWIZZLED)
-    w2c, w2s = nb.nvfp4_quantize(W2, False, g2, rt, nb.SF_SWIZZLED)
     H = torch.empty((M, N1), dtype=torch.float32, device=dev)
     Y = torch.empty((M, N2), dtype=torch.float32, device=dev)
-    nb.nvfp4_gemm(xc, xs, gx, w1c, w1s, g1, out=H)
+    Yf = torch.empty((M, N2), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(nb.nvfp4_linear_workspace_bytes(M, N1, K1, nb.LINEAR_FWD), nb.nvfp4_linear_workspace_bytes(M, N2, K2, nb.LINEAR_FWD)),
+                     dtype=torch.uint8, device=dev)
+    nb.nvfp4_linear_fwd(X, W1, nb.G_GIVEN, gx=gx, gw=g1, rx=rt, rw=rt, out=H, workspace=ws)
     gh = nb.nvfp4_tensor_amax_scale(H)              # the consumer's per-tensor scale must be known beforehand (delayed scaling)
     hc = torch.empty((M, N1 // 2), dtype=torch.uint8, device=dev)
     hs = torch.empty(nb.nvfp4_sf_bytes(M, N1, nb.SF_SWIZZLED), dtype=torch.uint8, device=dev)
-    L = nb.lib()
 
     def fused():
-        st = L.nvfp4_gemm_quantized(xc.data_ptr(), xs.data_ptr(), gx.data_ptr(), w1c.data_ptr(), w1s.data_ptr(), g1.data_ptr(),
-                                    M, N1, K1, gh.data_ptr(), C.byref(rt), hc.data_ptr(), hs.data_ptr(), nb.SF_SWIZZLED,
-                                    torch.cuda.current_stream().cuda_stream)
-        assert st == 0
-        nb.nvfp4_gemm(hc, hs, gh, w2c, w2s, g2, out=Y)
+        nb.nvfp4_linear_fwd_qout(X, W1, gy=gh, ry=rt, gscale_mode=nb.G_GIVEN, gx=gx, gw=g1, rx=rt, rw=rt, sf_layout=nb.SF_SWIZZLED,
+                                 codes=hc, scales=hs, workspace=ws)
+        nb.nvfp4_linear_fwd_qin(hc, hs, gh, W2, nb.G_GIVEN, gw=g2, rw=rt, out=Yf, workspace=ws)
 
-    def unfused():
-        nb.nvfp4_gemm(xc, xs, gx, w1c, w1s, g1, out=H)
-        nb.nvfp4_quantize(H, False, gh, rt, nb.SF_SWIZZLED, codes=hc, scales=hs)
-        nb.nvfp4_gemm(hc, hs, gh, w2c, w2s, g2, out=Y)
+    W2f = W2.float()                                # exact: the fp32 arm reads the same weight values
+    H16 = torch.empty((M, N1), dtype=torch.bfloat16, device=dev)
 
-    ms_f, ms_u = time_call(fused, 10), time_call(unfused, 10)
+    def unfused():                                  # fp32 intermediate: the same numbers as the fused arm, bit for bit
+        nb.nvfp4_linear_fwd(X, W1, nb.G_GIVEN, gx=gx, gw=g1, rx=rt, rw=rt, out=H, workspace=ws)
+        nb.nvfp4_linear_fwd(H, W2f, nb.G_GIVEN, gx=gh, gw=g2, rx=rt, rw=rt, out=Y, workspace=ws)
+
+    def unfused_bf16():                             # bf16 intermediate: half the bytes, one more rounding of H
+        nb.nvfp4_linear_fwd(X, W1, nb.G_GIVEN, gx=gx, gw=g1, rx=rt, rw=rt, out=H16, workspace=ws)
+        nb.nvfp4_linear_fwd(H16, W2, nb.G_GIVEN, gx=gh, gw=g2, rx=rt, rw=rt, out=Y, workspace=ws)
+
+    ms_f, ms_b, ms_u = time_call(fused, 10), time_call(unfused_bf16, 10), time_call(unfused, 10)
+    same = bool(torch.equal(Y, Yf))
     flops = 2.0 * M * (K1 * N1 + K2 * N2)
-    return {"workload": "up projection -> quantized in its epilogue -> down projection", "M": M, "K1": K1, "N1": N1, "N2": N2,
+    return {"workload": "up projection (nvfp4_linear_fwd_qout) -> down projection (nvfp4_linear_fwd_qin), given per-tensor scales",
+            "M": M, "K1": K1, "N1": N1, "N2": N2,
             "fused_ms": ms_f, "unfused_ms": ms_u, "time_saved_ms": ms_u - ms_f,
+            "unfused_bf16_intermediate_ms": ms_b, "time_saved_vs_bf16_intermediate_ms": ms_b - ms_f,
             "fused_TFLOPS": flops / ms_f / 1e9, "unfused_TFLOPS": flops / ms_u / 1e9,
+            "results_bit_identical_to_fp32_intermediate": same,
             "bytes_not_moved": M * N1 * 8,         # the fp32 intermediate is neither written nor read back
-            "bytes_note": "the M x N1 fp32 intermediate: 4 B/element written by the first GEMM + 4 B/element read by the quantizer"}
+            "bytes_note": "the M x N1 fp32 intermediate: 4 B/element written by the first GEMM + 4 B/element read by the next layer's quantizer"}
 
 
 def main():
@@ -483,9 +492,9 @@ def main():
     # ---- roofline of the dominant kernel (the GEMM): same workload, decomposed into the C-ABI's
     #      quantize and gemm calls so that CUDA events bracket every GEMM launch; clocks sampled meanwhile ----
     rt, sr = block.rt, block.sr
-    roof_sampler = ClockSampler(local).start() if rank == 0 else None
+    roof_sampler = ClockSampler(local, interval_s=0.002).start() if rank == 0 else None   # a short pass: sample it densely
     gemm_events, gemm_flops, gemm_bytes = [], 0.0, 0.0
-    roof_steps = min(args.steps, 6)
+    roof_steps = min(args.steps, 3)
     for it in range(roof_steps + 1):
         if it == 1 and roof_sampler is not None:
             torch.cuda.synchronize()

@@ -222,6 +222,32 @@ NVFP4_API int nvfp4_linear_bwd_dw(const void* dY, const void* X, int dtype, int6
                         void* dW, int dw_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
+ * Producer fusion along a chain of layers (Eq. 1 / Eq. 4 applied twice; in Section 5's model the position of
+ * the SwiGLU output feeding the down projection): the quantization Q(.) that the NEXT layer would apply to its
+ * input is done in the epilogue of the GEMM that produces it, so the intermediate never exists in bf16 or fp32.
+ *
+ * nvfp4_linear_fwd_qout: as nvfp4_linear_fwd, but instead of Y it writes Q(Y) with blocks of 16 along N
+ *   (y_codes [M, N/2], y_scales for the quantized shape (M, N) in `sf_layout`), using the per-tensor scale *gy
+ *   of the OUTPUT (device, NULL => 1; it has to be known before the product runs, e.g. carried over from the
+ *   previous step) and rounding ry (host).  Bit for bit what nvfp4_quantize makes of nvfp4_linear_fwd's fp32 Y.
+ *   N % 32 == 0.  Workspace as for nvfp4_linear_fwd.
+ * nvfp4_linear_fwd_qin: as nvfp4_linear_fwd for an input that is already quantized along K: x_codes [M, K/2],
+ *   x_scales in the swizzled layout, per-tensor scale *gx (device, NULL => 1), e.g. the output of
+ *   nvfp4_linear_fwd_qout with sf_layout = NVFP4_SF_SWIZZLED_128x4.  gscale_mode / gw / rw apply to W only.
+ *   Workspace: nvfp4_linear_workspace_bytes(M, N, K, NVFP4_LINEAR_FWD).
+ */
+NVFP4_API int nvfp4_linear_fwd_qout(const void* X, const void* W, int dtype, int64_t M, int64_t N, int64_t K,
+                          int gscale_mode, const float* gx, const float* gw,
+                          const nvfp4_rounding* rx, const nvfp4_rounding* rw,
+                          const float* gy, const nvfp4_rounding* ry /* host */,
+                          uint8_t* y_codes, uint8_t* y_scales, int sf_layout,
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+NVFP4_API int nvfp4_linear_fwd_qin(const uint8_t* x_codes, const uint8_t* x_scales, const float* gx,
+                         const void* W, int dtype, int64_t M, int64_t N, int64_t K,
+                         int gscale_mode, const float* gw, const nvfp4_rounding* rw,
+                         void* Y, int y_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
  * The layer of Eq. 1-6 with every tensor read once per pass (fused producers).
  *
  * Eq. 4-6 use X, W and dY in both orientations.  nvfp4_linear_fwd_save computes Y as

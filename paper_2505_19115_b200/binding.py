@@ -71,6 +71,10 @@ def lib():
     for name in ("nvfp4_linear_fwd", "nvfp4_linear_bwd_dx", "nvfp4_linear_bwd_dw"):
         getattr(L, name).restype = ci
         getattr(L, name).argtypes = lin
+    L.nvfp4_linear_fwd_qout.restype = ci
+    L.nvfp4_linear_fwd_qout.argtypes = [vp, vp, ci, i64, i64, i64, ci, vp, vp, rp, rp, vp, rp, vp, vp, ci, vp, sz, vp]
+    L.nvfp4_linear_fwd_qin.restype = ci
+    L.nvfp4_linear_fwd_qin.argtypes = [vp, vp, vp, vp, ci, i64, i64, i64, ci, vp, rp, vp, ci, vp, sz, vp]
     L.nvfp4_linear_saved_bytes.restype = sz
     L.nvfp4_linear_saved_bytes.argtypes = [i64, i64, i64]
     L.nvfp4_linear_fused_workspace_bytes.restype = sz
@@ -276,6 +280,45 @@ def nvfp4_linear_bwd_dw(dY, X, gscale_mode=G_AMAX, gdy=None, gx=None, rdy=None, 
     (M, N), K = dY.shape, X.shape[1]
     return _linear("nvfp4_linear_bwd_dw", LINEAR_BWD_DW, dY, X, M, N, K, (N, K), gscale_mode, gdy, gx,
                    rdy or Rounding(SR, 0, 1), rx or Rounding(SR, 0, 2), out, out_dtype, workspace, stream)
+
+
+def nvfp4_linear_fwd_qout(X, W, gy=None, ry=None, gscale_mode=G_AMAX, gx=None, gw=None, rx=None, rw=None,
+                          sf_layout=SF_SWIZZLED, codes=None, scales=None, workspace=None, stream=None):
+    """Forward layer whose output leaves the GEMM already quantized along N: returns (codes [M, N/2], scales)."""
+    (M, K), N = X.shape, W.shape[0]
+    if codes is None:
+        codes = torch.empty((M, N // 2), dtype=torch.uint8, device=X.device)
+    if scales is None:
+        if sf_layout == SF_LINEAR:
+            scales = torch.empty((M, N // 16), dtype=torch.uint8, device=X.device)
+        else:
+            scales = torch.empty(max(nvfp4_sf_bytes(M, N, sf_layout), 16), dtype=torch.uint8, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(nvfp4_linear_workspace_bytes(M, N, K, LINEAR_FWD), dtype=torch.uint8, device=X.device)
+    assert X.is_contiguous() and W.is_contiguous() and X.dtype == W.dtype
+    st = lib().nvfp4_linear_fwd_qout(_ptr(X), _ptr(W), _dtype_code(X), M, N, K, gscale_mode, _ptr(gx), _ptr(gw),
+                                     C.byref(rx or Rounding(RTN)), C.byref(rw or Rounding(RTN)), _ptr(gy),
+                                     C.byref(ry or Rounding(RTN)), _ptr(codes), _ptr(scales), sf_layout,
+                                     _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(st, "nvfp4_linear_fwd_qout")
+    return codes, scales
+
+
+def nvfp4_linear_fwd_qin(x_codes, x_scales, gx, W, gscale_mode=G_AMAX, gw=None, rw=None, out=None,
+                         out_dtype=torch.float32, workspace=None, stream=None):
+    """Forward layer for an input already quantized along K (codes [M, K/2], swizzled scales, per-tensor scale gx)."""
+    M, K = x_codes.shape[0], x_codes.shape[1] * 2
+    N = W.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=W.device)
+    if workspace is None:
+        workspace = torch.empty(nvfp4_linear_workspace_bytes(M, N, K, LINEAR_FWD), dtype=torch.uint8, device=W.device)
+    assert W.is_contiguous() and out.is_contiguous()
+    st = lib().nvfp4_linear_fwd_qin(_ptr(x_codes), _ptr(x_scales), _ptr(gx), _ptr(W), _dtype_code(W), M, N, K, gscale_mode,
+                                    _ptr(gw), C.byref(rw or Rounding(RTN)), _ptr(out), _dtype_code(out), _ptr(workspace),
+                                    workspace.numel(), _stream(stream))
+    _check(st, "nvfp4_linear_fwd_qin")
+    return out
 
 
 FUSED_FWD_SAVE, FUSED_BWD_SAVED, FUSED_BWD = 0, 1, 2

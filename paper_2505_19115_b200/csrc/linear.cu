@@ -59,6 +59,9 @@ int run_linear(int which, const void* a, const void* b, int dtype, int64_t M, in
   if (out_dtype != NVFP4_BF16 && out_dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
   if (gscale_mode != NVFP4_G_NONE && gscale_mode != NVFP4_G_AMAX && gscale_mode != NVFP4_G_GIVEN) return NVFP4_ERR_ENUM;
   if (gscale_mode == NVFP4_G_GIVEN && (!ga || !gb)) return NVFP4_ERR_NULL;
+  for (const nvfp4_rounding* r : {ra, rb})              // rejected here, before the amax launches, not by the quantizer after them
+    if ((r->mode != NVFP4_RTN && r->mode != NVFP4_SR) || r->reserved != 0) return NVFP4_ERR_ENUM;
+  if (!aligned16(a) || !aligned16(b) || !aligned16(out)) return NVFP4_ERR_ALIGN;
   Plan pl;
   if (!make_plan(M, N, K, which, &pl)) return NVFP4_ERR_SHAPE;
   if (!plan_ok(pl)) return NVFP4_ERR_SHAPE;
@@ -119,6 +122,76 @@ extern "C" int nvfp4_linear_bwd_dw(const void* dY, const void* X, int dtype, int
                                    void* dW, int dw_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream) {
   return run_linear(NVFP4_LINEAR_BWD_DW, dY, X, dtype, M, N, K, gscale_mode, gdy, gx, rdy, rx, dW, dw_dtype,
                     workspace, workspace_bytes, cuda_stream);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Producer fusion along a chain of layers (no high-precision round trip between them): the first layer
+// writes Q(Y) straight from its GEMM epilogue, the next layer takes that quantized operand as its Q(X).
+// ------------------------------------------------------------------------------------------------
+extern "C" int nvfp4_linear_fwd_qout(const void* X, const void* W, int dtype, int64_t M, int64_t N, int64_t K,
+                                     int gscale_mode, const float* gx, const float* gw,
+                                     const nvfp4_rounding* rx, const nvfp4_rounding* rw,
+                                     const float* gy, const nvfp4_rounding* ry,
+                                     uint8_t* y_codes, uint8_t* y_scales, int sf_layout,
+                                     void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!X || !W || !rx || !rw || !ry || !y_codes || !y_scales) return NVFP4_ERR_NULL;
+  if (dtype != NVFP4_BF16 && dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if (sf_layout != NVFP4_SF_LINEAR && sf_layout != NVFP4_SF_SWIZZLED_128x4) return NVFP4_ERR_ENUM;
+  for (const nvfp4_rounding* r : {rx, rw, ry})          // everything the later calls would reject is rejected before the first launch
+    if ((r->mode != NVFP4_RTN && r->mode != NVFP4_SR) || r->reserved != 0) return NVFP4_ERR_ENUM;
+  if (!aligned16(X) || !aligned16(W) || !aligned16(y_codes) || !aligned16(y_scales)) return NVFP4_ERR_ALIGN;
+  if (gscale_mode != NVFP4_G_NONE && gscale_mode != NVFP4_G_AMAX && gscale_mode != NVFP4_G_GIVEN) return NVFP4_ERR_ENUM;
+  if (gscale_mode == NVFP4_G_GIVEN && (!gx || !gw)) return NVFP4_ERR_NULL;
+  Plan pl;
+  if (!make_plan(M, N, K, NVFP4_LINEAR_FWD, &pl) || !plan_ok(pl) || N % 32 != 0) return NVFP4_ERR_SHAPE;
+  const Layout l = make_layout(pl);
+  if (!workspace || workspace_bytes < l.total || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return NVFP4_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  const float* g_x = nullptr;
+  const float* g_w = nullptr;
+  int st;
+  if (gscale_mode == NVFP4_G_AMAX) {
+    float* wa = reinterpret_cast<float*>(ws + l.a_g);
+    float* wb = reinterpret_cast<float*>(ws + l.b_g);
+    if ((st = nvfp4_tensor_amax_scale(X, dtype, M, K, K, wa, cuda_stream))) return st;
+    if ((st = nvfp4_tensor_amax_scale(W, dtype, N, K, K, wb, cuda_stream))) return st;
+    g_x = wa; g_w = wb;
+  } else if (gscale_mode == NVFP4_G_GIVEN) {
+    g_x = gx; g_w = gw;
+  }
+  if ((st = nvfp4_quantize(X, dtype, M, K, K, 0, g_x, rx, ws + l.a_codes, ws + l.a_sf, NVFP4_SF_SWIZZLED_128x4, cuda_stream))) return st;
+  if ((st = nvfp4_quantize(W, dtype, N, K, K, 0, g_w, rw, ws + l.b_codes, ws + l.b_sf, NVFP4_SF_SWIZZLED_128x4, cuda_stream))) return st;
+  return nvfp4_gemm_quantized(ws + l.a_codes, ws + l.a_sf, g_x, ws + l.b_codes, ws + l.b_sf, g_w, M, N, K, gy, ry, y_codes,
+                              y_scales, sf_layout, cuda_stream);
+}
+
+extern "C" int nvfp4_linear_fwd_qin(const uint8_t* x_codes, const uint8_t* x_scales, const float* gx,
+                                    const void* W, int dtype, int64_t M, int64_t N, int64_t K,
+                                    int gscale_mode, const float* gw, const nvfp4_rounding* rw,
+                                    void* Y, int y_dtype, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!x_codes || !x_scales || !W || !rw || !Y) return NVFP4_ERR_NULL;
+  if (dtype != NVFP4_BF16 && dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if ((rw->mode != NVFP4_RTN && rw->mode != NVFP4_SR) || rw->reserved != 0) return NVFP4_ERR_ENUM;
+  if (!aligned16(x_codes) || !aligned16(x_scales) || !aligned16(W) || !aligned16(Y)) return NVFP4_ERR_ALIGN;
+  if (y_dtype != NVFP4_BF16 && y_dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
+  if (gscale_mode != NVFP4_G_NONE && gscale_mode != NVFP4_G_AMAX && gscale_mode != NVFP4_G_GIVEN) return NVFP4_ERR_ENUM;
+  if (gscale_mode == NVFP4_G_GIVEN && !gw) return NVFP4_ERR_NULL;
+  Plan pl;
+  if (!make_plan(M, N, K, NVFP4_LINEAR_FWD, &pl) || !plan_ok(pl)) return NVFP4_ERR_SHAPE;
+  const Layout l = make_layout(pl);
+  if (!workspace || workspace_bytes < l.total || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return NVFP4_ERR_WORKSPACE;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  const float* g_w = nullptr;
+  int st;
+  if (gscale_mode == NVFP4_G_AMAX) {
+    float* wb = reinterpret_cast<float*>(ws + l.b_g);
+    if ((st = nvfp4_tensor_amax_scale(W, dtype, N, K, K, wb, cuda_stream))) return st;
+    g_w = wb;
+  } else if (gscale_mode == NVFP4_G_GIVEN) {
+    g_w = gw;
+  }
+  if ((st = nvfp4_quantize(W, dtype, N, K, K, 0, g_w, rw, ws + l.b_codes, ws + l.b_sf, NVFP4_SF_SWIZZLED_128x4, cuda_stream))) return st;
+  return nvfp4_gemm(x_codes, x_scales, gx, ws + l.b_codes, ws + l.b_sf, g_w, M, N, K, Y, y_dtype, N, cuda_stream);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -129,6 +129,16 @@ def test_newer_entry_points_reject_bad_arguments_on_the_host():
     bs = lambda **kw: L.nvfp4_linear_bwd_saved(kw.get("dY", buf), 0, 256, kw.get("N", 512), 512, 0, None, rb, rb, buf, 1 << 30,
                                                buf, 1, buf, kw.get("dwt", 1), kw.get("ws", buf), 1 << 30, None)
     assert bs(dY=None) == 1 and bs(N=500) == 2 and bs(dwt=7) == 4 and bs(ws=None) == 5
+    # chained layers: quantized output / quantized input
+    qo = lambda **kw: L.nvfp4_linear_fwd_qout(kw.get("X", buf), buf, 0, 256, kw.get("N", 512), kw.get("K", 512), kw.get("gm", 0), None, None,
+                                              rb, rb, None, kw.get("ry", rb), kw.get("yc", buf), buf, kw.get("sf", 1),
+                                              kw.get("ws", buf), 1 << 30, None)
+    assert qo(X=None) == 1 and qo(ry=None) == 1 and qo(yc=None) == 1 and qo(N=528) == 2 and qo(K=528) == 2
+    assert qo(gm=9) == 4 and qo(gm=2) == 1 and qo(ws=None) == 5 and qo(sf=5) == 4
+    qi = lambda **kw: L.nvfp4_linear_fwd_qin(kw.get("xc", buf), buf, None, kw.get("W", buf), 0, 256, 512, kw.get("K", 512), kw.get("gm", 0),
+                                             None, rb, buf, kw.get("yt", 1), kw.get("ws", buf), 1 << 30, None)
+    assert qi(xc=None) == 1 and qi(W=None) == 1 and qi(K=528) == 2 and qi(gm=9) == 4 and qi(gm=2) == 1
+    assert qi(yt=3) == 4 and qi(ws=None) == 5
     # quantized epilogue, bf16 and MXFP4 products, noise monitor, transpose
     gq = lambda **kw: L.nvfp4_gemm_quantized(kw.get("a", buf), buf, None, buf, buf, None, 128, kw.get("N", 128), 256, None,
                                              kw.get("r", rb), buf, buf, kw.get("sf", 0), None)

@@ -185,3 +185,41 @@ def test_non_finite_input_propagates_through_the_per_tensor_scale(bad):
     # the oracle's dequantize-then-matmul says the same
     ref, _ = oracle_linear("fwd", Xd, Wd, nb.Rounding(nb.RTN), nb.Rounding(nb.RTN), True)
     assert np.all(np.isnan(ref))
+
+
+# ---------------------------------------------------------------- a chain of layers without a high-precision intermediate
+@pytest.mark.parametrize("mode", [nb.RTN, nb.SR])
+@pytest.mark.parametrize("shape", [(256, 512, 768, 256), (300, 288, 544, 200)])
+def test_chained_layers_quantize_in_the_producer(shape, mode):
+    # layer 1 writes Q(H) from its GEMM epilogue (nvfp4_linear_fwd_qout), layer 2 consumes it (nvfp4_linear_fwd_qin).
+    # H itself (layer 1 through nvfp4_linear_fwd) is checked against the oracle's product; the quantized H must then
+    # be the ORACLE's quantization of that H byte for byte, and the second product the oracle's product of those codes.
+    M, K1, N1, N2 = shape
+    X, W1, _ = synth.linear_inputs(M, K1, N1, seed=41)
+    _, W2, _ = synth.linear_inputs(M, N1, N2, seed=42)
+    X, W1, W2 = X.cuda(), W1.cuda(), W2.cuda()
+    rt, ry = nb.Rounding(nb.RTN), nb.Rounding(mode, 77, 4)
+    H = nb.nvfp4_linear_fwd(X, W1, rx=rt, rw=rt)
+    ref, T = oracle_linear("fwd", X, W1, rt, rt, True)
+    Hh = _host(H)
+    _assert_close(Hh, ref, T)
+    gh_t = nb.nvfp4_tensor_amax_scale(H)                  # the consumer's scale has to be known beforehand
+    gh = ob.tensor_amax_scale(Hh)
+    assert np.float32(gh) == np.float32(gh_t.item())
+    hc, hs = nb.nvfp4_linear_fwd_qout(X, W1, gy=gh_t, ry=ry, rx=rt, rw=rt, sf_layout=nb.SF_SWIZZLED)
+    Y = nb.nvfp4_linear_fwd_qin(hc, hs, gh_t, W2, rw=rt)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
+    oc, osf = ob.quantize(Hh, g=gh, mode=ry.mode, seed=ry.seed, offset=ry.offset)
+    assert np.array_equal(hc.cpu().numpy(), oc)
+    assert np.array_equal(hs.cpu().numpy().reshape(-1), ob.sf_swizzle(osf).reshape(-1))
+    w2h = _host(W2)
+    g2 = ob.tensor_amax_scale(w2h)
+    wc, wsf = ob.quantize(w2h, g=g2)
+    ref2, T2 = ob.gemm(oc, osf, gh, wc, wsf, g2)
+    _assert_close(_host(Y), ref2, T2)
+    # and the unfused pair (fp32 H, quantized by the next layer's own quantizer) gives the same bits when the
+    # roundings agree (the next layer would use RtN on its input, Eq. 4)
+    if mode == nb.RTN:
+        Y_unfused = nb.nvfp4_linear_fwd(H, W2.float(), gscale_mode=nb.G_AMAX, rx=rt, rw=rt)   # bf16 -> fp32 is exact
+        assert torch.equal(Y, Y_unfused)
