@@ -293,8 +293,10 @@ NVFP4_API int nvfp4_linear_bwd(const void* dY, const void* W, const void* X, int
  * linear [Rq, Kq/32] or in the same 128-row x 4-block tiles of 512 bytes (a tile then covers 128
  * values); nvfp4_sf_bytes_mx gives the size.  The random integers of SR belong to groups of 16
  * elements exactly as for NVFP4 (group index r*(Kq/16) + k/16).  Kq % 32 == 0.
- * nvfp4_quantize_mx: transposed == 1 (bf16 only) transposes into `workspace` (rows*cols*2 bytes,
- * 16-byte aligned) and quantizes the rows of the transpose; workspace may be NULL otherwise.
+ * nvfp4_quantize_mx: transposed == 1 (bf16 only) quantizes along the rows straight from the source
+ * tile (no transpose pass, `workspace` unused and may be NULL); only a tensor with more than 2^24 rows
+ * goes through a transpose into `workspace` (rows*cols*2 bytes, 16-byte aligned) and is rejected with
+ * NVFP4_ERR_WORKSPACE without one.
  * nvfp4_gemm_mx: as nvfp4_gemm on MXFP4 operands (tcgen05 kind::mxf4, scale_vec::2X).
  */
 NVFP4_API size_t nvfp4_sf_bytes_mx(int64_t Rq, int64_t Kq, int sf_layout);

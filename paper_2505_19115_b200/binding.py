@@ -406,10 +406,13 @@ def nvfp4_quantize_mx(x, transposed: bool = False, global_scale=None, rounding: 
         scales = torch.empty((Rq, Kq // 32), dtype=torch.uint8, device=x.device)
     else:
         scales = torch.empty(max(nvfp4_sf_bytes_mx(Rq, Kq, sf_layout), 16), dtype=torch.uint8, device=x.device)
-    ws = torch.empty(rows * cols * 2, dtype=torch.uint8, device=x.device) if transposed else None
-    st = lib().nvfp4_quantize_mx(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), int(transposed), _ptr(global_scale),
-                                 C.byref(rounding), _ptr(codes), _ptr(scales), sf_layout, _ptr(ws),
-                                 ws.numel() if ws is not None else 0, _stream(stream))
+    def call(ws):
+        return lib().nvfp4_quantize_mx(_ptr(x), _dtype_code(x), rows, cols, x.stride(0), int(transposed), _ptr(global_scale),
+                                       C.byref(rounding), _ptr(codes), _ptr(scales), sf_layout, _ptr(ws),
+                                       ws.numel() if ws is not None else 0, _stream(stream))
+    st = call(None)
+    if st == 5 and transposed:          # a shape the tile kernel does not take: the library transposes into a workspace first
+        st = call(torch.empty(rows * cols * 2, dtype=torch.uint8, device=x.device))
     _check(st, "nvfp4_quantize_mx")
     return codes, scales
 

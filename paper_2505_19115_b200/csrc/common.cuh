@@ -38,7 +38,8 @@ inline cudaError_t set_max_dynamic_smem(DeviceFlags& flags, Kernel kernel, int b
 bool tile_quantizer_eligible(int dtype, int64_t rows, int64_t cols, bool dual);
 int tile_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, const float* g, bool dual,
                   const nvfp4_rounding* rt, uint8_t* codes_t, uint8_t* scales_t,
-                  const nvfp4_rounding* rr, uint8_t* codes_r, uint8_t* scales_r, int sf_layout, cudaStream_t s);
+                  const nvfp4_rounding* rr, uint8_t* codes_r, uint8_t* scales_r, int sf_layout, cudaStream_t s,
+                  bool mx_t = false);   // mx_t: MXFP4 (blocks of 32, E8M0 scales) for the transposed output, no row output
 int tile_error_word(unsigned int* out);
 
 // Per-tensor scale g = amax/2688 in one launch (quantize.cu); scratch_zeroed: two zeroed 32-bit device words.

@@ -468,10 +468,17 @@ extern "C" int nvfp4_quantize_mx(const void* x, int dtype, int64_t rows, int64_t
   if (Kq % 32 != 0 || rows >= (int64_t)1 << 31 || cols >= (int64_t)1 << 31) return NVFP4_ERR_SHAPE;
   if (!aligned16(x) || !aligned16(codes) || !aligned16(scales) || (ld % 8) != 0) return NVFP4_ERR_ALIGN;
   if (ceil_div(Rq, 128) > 65535) return NVFP4_ERR_SHAPE;
-  if (transposed && (!workspace || workspace_bytes < (size_t)rows * cols * 2 || (reinterpret_cast<uintptr_t>(workspace) & 15u)))
+  // bf16 tensors whose row count is a multiple of 32 (always true here: Kq = rows) go through the tile kernel, which
+  // quantizes along the rows straight from the source; the transpose pass remains for what that kernel does not take
+  const bool tile_path = transposed && rows % 32 == 0 && tile_quantizer_eligible(dtype, rows, cols, false);
+  if (transposed && !tile_path &&
+      (!workspace || workspace_bytes < (size_t)rows * cols * 2 || (reinterpret_cast<uintptr_t>(workspace) & 15u)))
     return NVFP4_ERR_WORKSPACE;
   if (int st = check_arch()) return st;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (tile_path)
+    return tile_quantize(x, rows, cols, ld, global_scale, false, rounding, codes, scales, nullptr, nullptr, nullptr, sf_layout, s,
+                         /*mx_t=*/true);
   const void* src = x;
   int64_t src_ld = ld;
   if (transposed) {

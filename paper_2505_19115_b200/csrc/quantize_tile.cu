@@ -33,7 +33,8 @@ struct TileParams {
   // transposed output (always): quantized shape (cols, rows)
   PhiloxStream t_rng;
   uint8_t* t_scales;
-  int64_t t_nkb, t_k_tiles;
+  int64_t t_nkb, t_k_tiles;   // groups of 16 per quantized row (the unit of the random draws); scale tiles per quantized row
+  int64_t t_nsb;              // scale blocks per quantized row: rows / 16 (NVFP4) or rows / 32 (MXFP4)
   // row output (DUAL only): quantized shape (rows, cols)
   PhiloxStream r_rng;
   uint8_t* r_scales;
@@ -49,7 +50,10 @@ __device__ __forceinline__ uint32_t swz128(uint32_t row, uint32_t byte) {
   return row * 128u + ((((byte >> 4) ^ (row & 7u)) << 4) | (byte & 15u));
 }
 
-template <bool SR_T, bool DUAL, bool SR_R, bool SWZ>
+// MX_T: the transposed output is MXFP4 (Section 3, Table 1): blocks of 32 rows with an E8M0 scale rounded up to a
+// power of two; a warp then takes 32 rows at a time, and the two groups of 16 inside a block keep their own
+// random draws (group index as for NVFP4).
+template <bool SR_T, bool DUAL, bool SR_R, bool SWZ, bool MX_T = false>
 __global__ void __launch_bounds__(kThreads, 4)
 quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_ct,
                      const __grid_constant__ CUtensorMap map_cr, const TileParams p) {
@@ -60,8 +64,9 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   uint8_t* codes_r = codes_t + kCodesTBytes;              // [256][32 B]
   uint8_t* sf_t = codes_r + kCodesRBytes;                 // [16][64]
   uint8_t* sf_r = sf_t + kSfTBytes;                       // [2][512]
+  static_assert(!(MX_T && DUAL), "the MXFP4 variant writes the transposed output only");
   __shared__ __align__(8) uint64_t bar;
-  __shared__ float inv_table[128];
+  __shared__ float inv_table[MX_T ? 256 : 128];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t c0 = (int64_t)blockIdx.x * kTileCols;
@@ -76,7 +81,7 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(smem_addr(tile)), "l"(&map_x), "r"(smem_addr(&bar)), "r"((int)c0), "r"((int)r0) : "memory");
   }
-  build_inv_table(inv_table, g);
+  if constexpr (MX_T) build_inv_table_mx(inv_table, g); else build_inv_table(inv_table, g);
   __syncthreads();                                        // barrier initialised, table published
   {
     // bounded wait for the tile; on a timeout every thread leaves without storing anything
@@ -100,6 +105,41 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
   // ---- transposed output: lane -> columns (2*lane, 2*lane+1), warp -> row blocks ----
   // Codes are staged as [column][128 bytes] with the 128-byte swizzle the tiled store expects.
+  if constexpr (MX_T) {
+    const int rb = warp;                                      // 8 warps, 8 blocks of 32 rows
+    uint32_t w[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) w[j] = *reinterpret_cast<const uint32_t*>(tile + swz128(rb * 32 + j, 4 * lane));
+    uint32_t m[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) m[j] = absmax_bf16x2(w[2 * j], w[2 * j + 1]);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) m[j] = absmax_bf16x2(m[2 * j], m[2 * j + 1]);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) m[j] = absmax_bf16x2(m[2 * j], m[2 * j + 1]);
+    const uint32_t mm = absmax_bf16x2(absmax_bf16x2(m[0], m[1]), absmax_bf16x2(m[2], m[3])) & 0x7FFF7FFFu;
+    const uint32_t sfa = e8m0_encode_up(__fmul_rn(__uint_as_float(mm << 16), c));
+    const uint32_t sfb = e8m0_encode_up(__fmul_rn(__uint_as_float(mm & 0xFFFF0000u), c));
+    const float inv_a = inv_table[sfa], inv_b = inv_table[sfb];
+    const int64_t ca = c0 + 2 * lane;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float va[16], vb[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        va[j] = __uint_as_float(w[16 * h + j] << 16);
+        vb[j] = __uint_as_float(w[16 * h + j] & 0xFFFF0000u);
+      }
+      const int64_t kb = r0 / 16 + rb * 2 + h;                // group of 16 along the quantized row
+      uint32_t lo, hi;
+      encode_codes<SR_T>(va, inv_a, p.t_rng, (uint64_t)(ca * p.t_nkb + kb), lo, hi);
+      *reinterpret_cast<uint2*>(codes_t + swz128(2 * lane, (rb * 2 + h) * 8)) = make_uint2(lo, hi);
+      encode_codes<SR_T>(vb, inv_b, p.t_rng, (uint64_t)((ca + 1) * p.t_nkb + kb), lo, hi);
+      *reinterpret_cast<uint2*>(codes_t + swz128(2 * lane + 1, (rb * 2 + h) * 8)) = make_uint2(lo, hi);
+    }
+    sf_t[rb * kTileCols + 2 * lane] = (uint8_t)sfa;
+    sf_t[rb * kTileCols + 2 * lane + 1] = (uint8_t)sfb;
+  } else {
 #pragma unroll 1
   for (int rb = warp; rb < kTileRows / 16; rb += kThreads / 32) {
     uint32_t w[16];
@@ -126,6 +166,7 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     encode_block<SR_T>(vb, __uint_as_float(mm & 0xFFFF0000u), c, inv_table, p.t_rng, (uint64_t)((ca + 1) * p.t_nkb + kb), lo, hi, sf);
     *reinterpret_cast<uint2*>(codes_t + swz128(2 * lane + 1, rb * 8)) = make_uint2(lo, hi);
     sf_t[rb * kTileCols + 2 * lane + 1] = (uint8_t)sf;
+  }
   }
 
   // ---- row output: thread -> (row, block of 16 columns); four rows per thread ----
@@ -165,12 +206,15 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
   }
 
   // ---- scales out ----
-  const int64_t kb0 = r0 / 16;
+  constexpr int kSbRows = MX_T ? 32 : 16;                     // rows per scale block of the transposed output
+  constexpr int kSbPerTile = kTileRows / kSbRows;             // 16 or 8 scale blocks per column
+  constexpr int kKtPerTile = kSbPerTile / 4;                  // 4 or 2 scale tiles per column
+  const int64_t kb0 = r0 / kSbRows;
   if constexpr (SWZ) {
     // transposed scales: one 32-bit word = four row blocks of one column
     const bool fill_upper = ((c0 & 127) == 0) && (c0 + kTileCols >= p.cols);   // nobody else owns rows 64..127
-    for (int id = threadIdx.x; id < kTileCols * 4; id += kThreads) {
-      const int cl = id >> 2, t = id & 3;
+    for (int id = threadIdx.x; id < kTileCols * kKtPerTile; id += kThreads) {
+      const int cl = id / kKtPerTile, t = id % kKtPerTile;
       const int64_t kt = kb0 / 4 + t;
       if (kt >= p.t_k_tiles) continue;
       const uint8_t* s4 = sf_t + (t * 4) * kTileCols + cl;
@@ -191,9 +235,9 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
       }
     }
   } else {
-    for (int id = threadIdx.x; id < kTileCols * (kTileRows / 16); id += kThreads) {
-      const int cl = id >> 4, u = id & 15;
-      if (c0 + cl < p.cols && kb0 + u < p.t_nkb) p.t_scales[(c0 + cl) * p.t_nkb + kb0 + u] = sf_t[u * kTileCols + cl];
+    for (int id = threadIdx.x; id < kTileCols * kSbPerTile; id += kThreads) {
+      const int cl = id / kSbPerTile, u = id % kSbPerTile;
+      if (c0 + cl < p.cols && kb0 + u < p.t_nsb) p.t_scales[(c0 + cl) * p.t_nsb + kb0 + u] = sf_t[u * kTileCols + cl];
     }
   }
   if (threadIdx.x == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging must outlive the stores' reads
@@ -211,13 +255,13 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, const void* base, uin
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool SR_T, bool DUAL, bool SR_R, bool SWZ>
+template <bool SR_T, bool DUAL, bool SR_R, bool SWZ, bool MX_T = false>
 cudaError_t launch_tile(const CUtensorMap& mx, const CUtensorMap& mct, const CUtensorMap& mcr, const TileParams& p,
                         cudaStream_t s) {
   static DeviceFlags smem_set;   // per instantiation, per device
-  if (cudaError_t e = set_max_dynamic_smem(smem_set, quantize_tile_kernel<SR_T, DUAL, SR_R, SWZ>, kTileSmem)) return e;
+  if (cudaError_t e = set_max_dynamic_smem(smem_set, quantize_tile_kernel<SR_T, DUAL, SR_R, SWZ, MX_T>, kTileSmem)) return e;
   dim3 grid((unsigned)ceil_div(p.cols, kTileCols), (unsigned)ceil_div(p.rows, kTileRows));
-  quantize_tile_kernel<SR_T, DUAL, SR_R, SWZ><<<grid, kThreads, kTileSmem, s>>>(mx, mct, mcr, p);
+  quantize_tile_kernel<SR_T, DUAL, SR_R, SWZ, MX_T><<<grid, kThreads, kTileSmem, s>>>(mx, mct, mcr, p);
   return cudaGetLastError();
 }
 
@@ -246,7 +290,7 @@ bool tile_quantizer_eligible(int dtype, int64_t rows, int64_t cols, bool dual) {
 // Launches the tile kernel.  r_* arguments are ignored unless `dual`.  Arguments are validated by the callers.
 int tile_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, const float* g, bool dual,
                   const nvfp4_rounding* rt, uint8_t* codes_t, uint8_t* scales_t,
-                  const nvfp4_rounding* rr, uint8_t* codes_r, uint8_t* scales_r, int sf_layout, cudaStream_t s) {
+                  const nvfp4_rounding* rr, uint8_t* codes_r, uint8_t* scales_r, int sf_layout, cudaStream_t s, bool mx_t) {
   CUtensorMap mx, mct, mcr;
   if (!make_map_2d(&mx, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, x, (uint64_t)cols, (uint64_t)rows, (uint64_t)ld * 2, kTileCols,
                    kTileRows, CU_TENSOR_MAP_SWIZZLE_128B))
@@ -261,13 +305,21 @@ int tile_quantize(const void* x, int64_t rows, int64_t cols, int64_t ld, const f
   TileParams p;
   p.gptr = g; p.rows = rows; p.cols = cols;
   philox_stream_init(&p.t_rng, rt->seed, rt->offset);
-  p.t_scales = scales_t; p.t_nkb = rows / 16; p.t_k_tiles = ceil_div(p.t_nkb, 4);
+  p.t_scales = scales_t; p.t_nkb = rows / 16;
+  p.t_nsb = mx_t ? rows / 32 : rows / 16;
+  p.t_k_tiles = ceil_div(p.t_nsb, 4);
   const nvfp4_rounding* r2 = dual ? rr : rt;
   philox_stream_init(&p.r_rng, r2->seed, r2->offset);
   p.r_scales = scales_r; p.r_nkb = cols / 16; p.r_k_tiles = ceil_div(p.r_nkb, 4);
   const bool swz = sf_layout == NVFP4_SF_SWIZZLED_128x4;
   const bool sr_t = rt->mode == NVFP4_SR, sr_r = dual && rr->mode == NVFP4_SR;
   cudaError_t e;
+  if (mx_t) {                                                 // MXFP4, transposed output only
+    if (dual) return NVFP4_ERR_ENUM;
+    if (sr_t) e = swz ? launch_tile<true, false, false, true, true>(mx, mct, mcr, p, s) : launch_tile<true, false, false, false, true>(mx, mct, mcr, p, s);
+    else e = swz ? launch_tile<false, false, false, true, true>(mx, mct, mcr, p, s) : launch_tile<false, false, false, false, true>(mx, mct, mcr, p, s);
+    return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
+  }
   if (dual) e = swz ? dispatch_tile<true, true>(sr_t, sr_r, mx, mct, mcr, p, s) : dispatch_tile<true, false>(sr_t, sr_r, mx, mct, mcr, p, s);
   else e = swz ? dispatch_tile<false, true>(sr_t, sr_r, mx, mct, mcr, p, s) : dispatch_tile<false, false>(sr_t, sr_r, mx, mct, mcr, p, s);
   return e == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;

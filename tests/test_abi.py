@@ -147,9 +147,10 @@ def test_newer_entry_points_reject_bad_arguments_on_the_host():
     assert gb(a=None) == 1 and gb(K=24) == 2 and gb(dt=5) == 4 and gb(ldd=130) == 3
     gm = lambda **kw: L.nvfp4_gemm_mx(kw.get("a", buf), buf, None, buf, buf, None, 128, 128, kw.get("K", 256), buf, 1, 128, None)
     assert gm(a=None) == 1 and gm(K=48) == 2
-    qm = lambda **kw: L.nvfp4_quantize_mx(kw.get("x", buf), kw.get("dtype", 0), 32, kw.get("cols", 64), 64, kw.get("tr", 0), None, rb,
+    qm = lambda **kw: L.nvfp4_quantize_mx(kw.get("x", buf), kw.get("dtype", 0), kw.get("rows", 32), kw.get("cols", 64), 64, kw.get("tr", 0), None, rb,
                                           buf, buf, 0, kw.get("ws", None), 0, None)
-    assert qm(x=None) == 1 and qm(cols=48) == 2 and qm(tr=1, dtype=1) == 4 and qm(tr=1) == 5
+    assert qm(x=None) == 1 and qm(cols=48) == 2 and qm(tr=1, dtype=1) == 4
+    assert qm(tr=1, rows=1 << 25) == 5          # beyond the tile kernel's grid: needs the transpose workspace
     assert nb.nvfp4_sf_bytes_mx(128, 128, nb.SF_SWIZZLED) == 512 and nb.nvfp4_sf_bytes_mx(3, 64, nb.SF_LINEAR) == 6
     assert nb.nvfp4_sf_bytes_mx(3, 48, nb.SF_LINEAR) == 0
     nz = lambda **kw: L.nvfp4_quantization_noise(kw.get("x", buf), 0, 32, kw.get("cols", 32), 32, 0, None, buf, buf, 0,

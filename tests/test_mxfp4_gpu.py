@@ -38,16 +38,37 @@ def test_row_quantizer_matches_the_oracle(shape, mode, sf_layout, dtype):
         assert np.array_equal(scales.cpu().numpy().reshape(-1), want.reshape(-1))
 
 
+@pytest.mark.parametrize("sf_layout", [nb.SF_LINEAR, nb.SF_SWIZZLED])
 @pytest.mark.parametrize("mode", [nb.RTN, nb.SR])
-@pytest.mark.parametrize("shape", [(32, 8), (64, 72), (512, 200), (1056, 264)])
-def test_transposed_quantizer_matches_the_oracle(shape, mode):
+@pytest.mark.parametrize("shape", [(32, 8), (64, 72), (512, 200), (1056, 264), (288, 136), (2048, 1024)])
+def test_transposed_quantizer_matches_the_oracle(shape, mode, sf_layout):
+    # blocks of 32 along the rows, straight from the source tile (no transpose pass): ragged tiles in both directions
     x = synth.normal(shape, 1e-3, 4, device="cpu").cuda()
     g_t = nb.nvfp4_tensor_amax_scale(x)
     r = nb.Rounding(mode, 2, 1)
-    codes, scales = nb.nvfp4_quantize_mx(x, True, g_t, r, nb.SF_SWIZZLED)
+    codes, scales = nb.nvfp4_quantize_mx(x, True, g_t, r, sf_layout)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
     oc, osf = ob.quantize_mx(_h(x), g=float(g_t.item()), mode=mode, seed=2, offset=1, transposed=True)
     assert np.array_equal(codes.cpu().numpy(), oc)
-    assert np.array_equal(scales.cpu().numpy().reshape(-1), _swz(osf).reshape(-1))
+    want = _swz(osf) if sf_layout == nb.SF_SWIZZLED else osf
+    assert np.array_equal(scales.cpu().numpy().reshape(-1), want.reshape(-1))
+
+
+def test_transposed_special_blocks_and_no_global_scale():
+    x = torch.zeros((64, 16), dtype=torch.float32)
+    x[:8, 0] = torch.tensor([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0])   # amax 6 -> scale 1, the tie points
+    x[32:40, 1] = -x[:8, 0]
+    x[5, 2] = -0.0
+    x[0, 3] = 3.0                                                            # amax/6 = 0.5 exactly: a power of two
+    x[0, 4] = 3.0001
+    x[:32, 5] = 1e-30
+    x[40, 6] = 1e30
+    xs = x.to(torch.bfloat16).cuda()
+    for mode in (nb.RTN, nb.SR):
+        codes, scales = nb.nvfp4_quantize_mx(xs, True, None, nb.Rounding(mode, 3, 3), nb.SF_LINEAR)
+        oc, osf = ob.quantize_mx(_h(xs), mode=mode, seed=3, offset=3, transposed=True)
+        assert np.array_equal(codes.cpu().numpy(), oc) and np.array_equal(scales.cpu().numpy(), osf)
 
 
 def test_special_blocks():
