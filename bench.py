@@ -36,9 +36,9 @@ NOMINAL_FP4_TFLOPS = 9000.0
 MMA_FLOP_PER_CLK_PER_SM = 32768.0   # 2 * 256 * 256 * 64 FLOP per 128 cycles on a CTA pair (microbench mma_peak measures it)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM traffic of the GEMM kernel from the committed ncu capture (profiles/gemm2_nvfp4_kernel_8192x8192x4096.md):
-# 83.0 MB read + 212.2 MB written for 306.2 MB of algorithmic bytes (operand codes and scales + fp32 output).
+# 82.9 MB read + 211.2 MB written for 306.2 MB of algorithmic bytes (operand codes and scales + fp32 output).
 # GEMM traffic follows bytes, not FLOPs, so the workload's figure is this ratio times its own algorithmic bytes.
-GEMM_TRAFFIC_RATIO = (83.05 + 212.17) / 306.2
+GEMM_TRAFFIC_RATIO = (82.91 + 211.22) / 306.2
 
 
 def load_peaks():

@@ -140,7 +140,7 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     sf_t[rb * kTileCols + 2 * lane] = (uint8_t)sfa;
     sf_t[rb * kTileCols + 2 * lane + 1] = (uint8_t)sfb;
   } else {
-#pragma unroll 1
+#pragma unroll
   for (int rb = warp; rb < kTileRows / 16; rb += kThreads / 32) {
     uint32_t w[16];
 #pragma unroll
