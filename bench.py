@@ -428,6 +428,26 @@ def fused_producer_leg(nb, dev, cfg):
             "bytes_note": "the M x N1 fp32 intermediate: 4 B/element written by the first GEMM + 4 B/element read by the next layer's quantizer"}
 
 
+def qaf_backward_leg(nb, dev, cfg):
+    """The paper's fine-tuning phase (Section 5): forward in NVFP4, backward and update products in BF16.  The two BF16
+    products of the first layer, W, X and dY read as they are stored (MN-major operands, no transposed copies)."""
+    M = cfg["tokens"]
+    name, K, N = cfg["linears"][0]
+    X, W, dY = synth.linear_inputs(M, K, N, seed=4200, device=dev)
+    dX = torch.empty((M, K), dtype=torch.float32, device=dev)
+    dW = torch.empty((N, K), dtype=torch.float32, device=dev)
+    L = nb.lib()
+
+    def run():
+        st = L.nvfp4_linear_bwd_bf16(dY.data_ptr(), W.data_ptr(), X.data_ptr(), M, N, K, dX.data_ptr(), nb.FP32,
+                                     dW.data_ptr(), nb.FP32, None, 0, torch.cuda.current_stream().cuda_stream)
+        assert st == 0
+    ms = time_call(run, 10)
+    flops = 4.0 * M * N * K
+    return {"workload": f"layer '{name}' backward + update in bf16 (nvfp4_linear_bwd_bf16)", "M": M, "K": K, "N": N,
+            "ms": ms, "TFLOPS": flops / ms / 1e9}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -613,6 +633,8 @@ def main():
         configs["long_token_axis_weight_gradient"] = long_token_axis_leg(nb, dev)
         torch.cuda.empty_cache()
         configs["quantization_fused_into_producer"] = fused_producer_leg(nb, dev, synth.LLAMA_7B)
+        torch.cuda.empty_cache()
+        configs["qaf_backward_bf16"] = qaf_backward_leg(nb, dev, synth.LLAMA_7B)
         torch.cuda.empty_cache()
         err_word = nb.nvfp4_device_error_word()
         if err_word:

@@ -315,13 +315,19 @@ NVFP4_API int nvfp4_gemm_mx(const uint8_t* a_codes, const uint8_t* a_sf, const f
  * nvfp4_gemm_bf16: D[M,N] = A[M,K] . B[N,K]^T for dense bf16 A and B (both contiguous along K),
  * fp32 accumulation, D fp32 or bf16 with leading dimension ldd.  K % 16 == 0, pointers 16-byte
  * aligned, ldd*sizeof(D) a multiple of 16.
+ * nvfp4_gemm_bf16_ex: the same product for operands stored the other way round: a_mn_major == 1 means A is
+ * given as a dense [K, M] array (its output axis contiguous), b_mn_major == 1 means B is given as [K, N]; the
+ * tensor cores read them in place (no transposed copy).  M % 8 == 0 / N % 8 == 0 for such an operand.
+ * Combinations: (0,0), (0,1), (1,1) -- the three shapes the products of Eq. 1-3 take.
  * nvfp4_transpose_bf16: out[cols, rows] = x[rows, cols]^T (rows, cols multiples of 8; out dense).
  * nvfp4_linear_bwd_bf16: dX[M,K] = dY . W and dW[N,K] = dY^T . X from bf16 dY[M,N], W[N,K], X[M,K]
- * (all dense): transposes W, X and dY into the workspace (nvfp4_linear_bwd_bf16_workspace_bytes,
- * 256-byte aligned) and runs the two products.  M, N, K multiples of 16.
+ * (all dense), each read as it is stored.  `workspace` is unused (nvfp4_linear_bwd_bf16_workspace_bytes
+ * returns 0; NULL is accepted).  M, N, K multiples of 16.
  */
 NVFP4_API int nvfp4_gemm_bf16(const void* a, const void* b, int64_t M, int64_t N, int64_t K,
                     void* d, int d_dtype, int64_t ldd, void* cuda_stream);
+NVFP4_API int nvfp4_gemm_bf16_ex(const void* a, int a_mn_major, const void* b, int b_mn_major, int64_t M, int64_t N, int64_t K,
+                       void* d, int d_dtype, int64_t ldd, void* cuda_stream);
 NVFP4_API int nvfp4_transpose_bf16(const void* x, int64_t rows, int64_t cols, int64_t ld, void* out, void* cuda_stream);
 NVFP4_API size_t nvfp4_linear_bwd_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K);
 NVFP4_API int nvfp4_linear_bwd_bf16(const void* dY, const void* W, const void* X, int64_t M, int64_t N, int64_t K,

@@ -93,6 +93,8 @@ def lib():
     L.nvfp4_gemm_mx.argtypes = [vp, vp, vp, vp, vp, vp, i64, i64, i64, vp, ci, i64, vp]
     L.nvfp4_gemm_bf16.restype = ci
     L.nvfp4_gemm_bf16.argtypes = [vp, vp, i64, i64, i64, vp, ci, i64, vp]
+    L.nvfp4_gemm_bf16_ex.restype = ci
+    L.nvfp4_gemm_bf16_ex.argtypes = [vp, ci, vp, ci, i64, i64, i64, vp, ci, i64, vp]
     L.nvfp4_transpose_bf16.restype = ci
     L.nvfp4_transpose_bf16.argtypes = [vp, i64, i64, i64, vp, vp]
     L.nvfp4_linear_bwd_bf16_workspace_bytes.restype = sz
@@ -437,6 +439,18 @@ def nvfp4_gemm_bf16(A, B, out_dtype=torch.float32, out=None, stream=None):
         out = torch.empty((M, N), dtype=out_dtype, device=A.device)
     _check(lib().nvfp4_gemm_bf16(_ptr(A), _ptr(B), M, N, K, _ptr(out), _dtype_code(out), out.stride(0), _stream(stream)),
            "nvfp4_gemm_bf16")
+    return out
+
+
+def nvfp4_gemm_bf16_ex(A, a_mn_major, B, b_mn_major, out_dtype=torch.float32, out=None, stream=None):
+    """D[M,N] = A . B^T on bf16 operands; an MN-major operand is passed as its stored [K, M] (or [K, N]) array."""
+    assert A.dtype == torch.bfloat16 and B.dtype == torch.bfloat16 and A.is_contiguous() and B.is_contiguous()
+    (K, M) = A.shape if a_mn_major else A.shape[::-1]
+    N = B.shape[1] if b_mn_major else B.shape[0]
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=A.device)
+    _check(lib().nvfp4_gemm_bf16_ex(_ptr(A), int(a_mn_major), _ptr(B), int(b_mn_major), M, N, K, _ptr(out), _dtype_code(out),
+                                    out.stride(0), _stream(stream)), "nvfp4_gemm_bf16_ex")
     return out
 
 

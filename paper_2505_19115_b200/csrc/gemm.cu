@@ -422,13 +422,19 @@ struct Gemm2Params {
 // MX: MXFP4 operands (blocks of 32, E8M0 scales): a 512-byte scale tile then covers 128 values, a
 // stage holds two tiles per 128 rows instead of four, and two consecutive instructions share a
 // scale column, each using one half of it.
-template <int BN, int OUT, bool BF16_IN = false, bool MX = false>
+// MN (bf16 operands only): bit 0 / bit 1 = operand A / B is stored with its OUTPUT axis contiguous, [K, M] or [K, N]
+// row-major, instead of [M, K] / [N, K] (the backward and update products of Eq. 2-3 read W, X and dY that way): a
+// stage then holds, per operand, two boxes of 64 contraction rows x 64 output rows (128 bytes), and the MMA reads
+// them through MN-major descriptors, so no transposed copy of the tensor is ever made.
+template <int BN, int OUT, bool BF16_IN = false, bool MX = false, int MN = 0>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemm2Threads, 1)
 gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                    const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb,
                    const __grid_constant__ CUtensorMap map_d, const Gemm2Params p) {
   using C = Cfg2<BN>;
   constexpr bool BF16_OUT = (OUT == 1), Q_OUT = (OUT == 2);
+  constexpr bool MN_A = (MN & 1) != 0, MN_B = (MN & 2) != 0;
+  static_assert(MN == 0 || (BF16_IN && BN == 256), "MN-major operands exist for the bf16 variant with the 256-wide tile");
   static_assert(!Q_OUT || BN == 256, "the quantized epilogue stores one 128-byte row of codes per tile row");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -498,8 +504,18 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
         const uint32_t lead_full = map_to_cta(full_bar(s), 0);
         if (issuer) {
           if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2u * kOperandTx);
-          tma_load_2d_pair(st, &map_a, lead_full, ks * BK_BYTES, m0);
-          tma_load_2d_pair(st + C::kABytes, &map_b, lead_full, ks * BK_BYTES, n0);
+          if constexpr (MN_A) {                     // [K, M]: x = byte offset of the output row, y = contraction index
+            tma_load_2d_pair(st, &map_a, lead_full, m0 * 2, ks * 64);
+            tma_load_2d_pair(st + C::kABytes / 2, &map_a, lead_full, (m0 + 64) * 2, ks * 64);
+          } else {
+            tma_load_2d_pair(st, &map_a, lead_full, ks * BK_BYTES, m0);
+          }
+          if constexpr (MN_B) {
+            tma_load_2d_pair(st + C::kABytes, &map_b, lead_full, n0 * 2, ks * 64);
+            tma_load_2d_pair(st + C::kABytes + C::kBBytes / 2, &map_b, lead_full, (n0 + 64) * 2, ks * 64);
+          } else {
+            tma_load_2d_pair(st + C::kABytes, &map_b, lead_full, ks * BK_BYTES, n0);
+          }
         }
         if (++s == C::kStages) { s = 0; ph ^= 1u; }
       }
@@ -547,7 +563,7 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     // ------------------------------- MMA issuer (leader CTA only) -------------------------------
     if (rank == 0) {
       const bool issuer = elect_one();
-      constexpr uint32_t idesc = BF16_IN ? instr_desc_bf16(256, BN) : instr_desc(256, BN);
+      constexpr uint32_t idesc = BF16_IN ? instr_desc_bf16(256, BN, MN_A, MN_B) : instr_desc(256, BN);
       int s = 0, b = 0, acc = 0;
       uint32_t ph = 0, bph = 0, acc_ph = 0;
       bool ok = true;
@@ -571,9 +587,12 @@ gemm2_nvfp4_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
           const int nkt = min(4, p.k_mmas - ks * 4);
           const uint32_t sfa_t = tmem_base + C::kSfaCol + b * C::kSfCols;
           const uint32_t sfb_t = sfa_t + 16 + sfb_off;
-          const uint64_t adesc = operand_desc(st), bdesc = operand_desc(st + C::kABytes);
+          const uint64_t adesc = MN_A ? operand_desc_mn(st, C::kABytes / 2) : operand_desc(st);
+          const uint64_t bdesc = MN_B ? operand_desc_mn(st + C::kABytes, C::kBBytes / 2) : operand_desc(st + C::kABytes);
           if (issuer && BF16_IN) {
-            for (int j = 0; j < nkt; ++j) tc_mma_bf16_pair(d_tmem, adesc + 2u * j, bdesc + 2u * j, idesc, (ks | j) ? 1u : 0u);
+            // one instruction = 16 contraction indices: 32 bytes along a K-major row, 16 rows (2048 bytes) of an MN-major box
+            constexpr uint32_t a_step = MN_A ? (2048u >> 4) : 2u, b_step = MN_B ? (2048u >> 4) : 2u;
+            for (int j = 0; j < nkt; ++j) tc_mma_bf16_pair(d_tmem, adesc + a_step * j, bdesc + b_step * j, idesc, (ks | j) ? 1u : 0u);
             tc_commit_pair(empty_bar(s));
           } else if (issuer && MX) {
             for (int j = 0; j < nkt; ++j)
@@ -928,14 +947,17 @@ bool make_qout_map(CUtensorMap* map, uint8_t* base, int64_t M, int64_t N) {
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int OUT, bool BF16_IN = false, bool MX = false>
+template <int BN, int OUT, bool BF16_IN = false, bool MX = false, int MN = 0>
 int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParams& g, cudaStream_t s,
                  const QuantOut& q = QuantOut()) {
   using C = Cfg2<BN>;
   CUtensorMap map_a, map_b, map_sfa, map_sfb, map_d;
   const int64_t row_bytes = BF16_IN ? (int64_t)g.K * 2 : g.K / 2;       // operand rows as bytes
-  if (!make_codes_map(&map_a, a_codes, g.M, row_bytes, 128)) return NVFP4_ERR_CUDA;
-  if (!make_codes_map(&map_b, b_codes, g.N, row_bytes, BN / 2)) return NVFP4_ERR_CUDA;
+  // MN-major bf16 operand: the tensor is [K, rows] with the output axis contiguous; boxes of 64 contraction rows x 128 bytes
+  if (!((MN & 1) ? make_codes_map(&map_a, a_codes, g.K, (int64_t)g.M * 2, 64) : make_codes_map(&map_a, a_codes, g.M, row_bytes, 128)))
+    return NVFP4_ERR_CUDA;
+  if (!((MN & 2) ? make_codes_map(&map_b, b_codes, g.K, (int64_t)g.N * 2, 64) : make_codes_map(&map_b, b_codes, g.N, row_bytes, BN / 2)))
+    return NVFP4_ERR_CUDA;
   if constexpr (BF16_IN) {
     map_sfa = map_a;                                                     // never used by the kernel
     map_sfb = map_b;
@@ -960,12 +982,12 @@ int launch_gemm2(const uint8_t* a_codes, const uint8_t* b_codes, const GemmParam
   philox_stream_init(&p.out_rng, q.rounding ? q.rounding->seed : 0, q.rounding ? q.rounding->offset : 0);
   if (q.rounding) p.out_sr = q.rounding->mode == NVFP4_SR;
   static DeviceFlags smem_set;                         // per instantiation, per device
-  if (set_max_dynamic_smem(smem_set, gemm2_nvfp4_kernel<BN, OUT, BF16_IN, MX>, C::kSmemBytes) != cudaSuccess)
+  if (set_max_dynamic_smem(smem_set, gemm2_nvfp4_kernel<BN, OUT, BF16_IN, MX, MN>, C::kSmemBytes) != cudaSuccess)
     return NVFP4_ERR_CUDA;
   const int tiles = p.tiles_m * p.tiles_n;
   const int max_pairs = sm_count() / 2;
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  gemm2_nvfp4_kernel<BN, OUT, BF16_IN, MX><<<2 * pairs, kGemm2Threads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
+  gemm2_nvfp4_kernel<BN, OUT, BF16_IN, MX, MN><<<2 * pairs, kGemm2Threads, C::kSmemBytes, s>>>(map_a, map_b, map_sfa, map_sfb, map_d, p);
   return cudaGetLastError() == cudaSuccess ? NVFP4_OK : NVFP4_ERR_CUDA;
 }
 
@@ -1082,9 +1104,28 @@ extern "C" int nvfp4_gemm_mx(const uint8_t* a_codes, const uint8_t* a_sf, const 
                      : launch_gemm2<256, 0, false, true>(a_codes, b_codes, p, s);
 }
 
+namespace {
+int gemm_bf16_any(const void* a, int a_mn, const void* b, int b_mn, int64_t M, int64_t N, int64_t K,
+                  void* d, int d_dtype, int64_t ldd, void* cuda_stream);
+}
+
 extern "C" int nvfp4_gemm_bf16(const void* a, const void* b, int64_t M, int64_t N, int64_t K,
                                void* d, int d_dtype, int64_t ldd, void* cuda_stream) {
+  return gemm_bf16_any(a, 0, b, 0, M, N, K, d, d_dtype, ldd, cuda_stream);
+}
+
+extern "C" int nvfp4_gemm_bf16_ex(const void* a, int a_mn_major, const void* b, int b_mn_major, int64_t M, int64_t N, int64_t K,
+                                  void* d, int d_dtype, int64_t ldd, void* cuda_stream) {
+  if ((a_mn_major != 0 && a_mn_major != 1) || (b_mn_major != 0 && b_mn_major != 1)) return NVFP4_ERR_ENUM;
+  if (a_mn_major && !b_mn_major) return NVFP4_ERR_ENUM;      // no product of Eq. 1-3 has that shape; not instantiated
+  return gemm_bf16_any(a, a_mn_major, b, b_mn_major, M, N, K, d, d_dtype, ldd, cuda_stream);
+}
+
+namespace {
+int gemm_bf16_any(const void* a, int a_mn, const void* b, int b_mn, int64_t M, int64_t N, int64_t K,
+                  void* d, int d_dtype, int64_t ldd, void* cuda_stream) {
   if (!a || !b || !d) return NVFP4_ERR_NULL;
+  if ((a_mn && M % 8 != 0) || (b_mn && N % 8 != 0)) return NVFP4_ERR_SHAPE;   // 16-byte row pitch of an MN-major operand
   if (d_dtype != NVFP4_BF16 && d_dtype != NVFP4_FP32) return NVFP4_ERR_ENUM;
   if (M <= 0 || N <= 0 || K <= 0 || (K % 16) != 0 || ldd < N) return NVFP4_ERR_SHAPE;
   if (M >= (1ll << 31) - 256 || N >= (1ll << 31) - 256 || K >= (1ll << 30)) return NVFP4_ERR_SHAPE;
@@ -1104,8 +1145,15 @@ extern "C" int nvfp4_gemm_bf16(const void* a, const void* b, int64_t M, int64_t 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const uint8_t* ab = static_cast<const uint8_t*>(a);
   const uint8_t* bb = static_cast<const uint8_t*>(b);
-  return p.d_is_bf16 ? launch_gemm2<256, 1, true>(ab, bb, p, s) : launch_gemm2<256, 0, true>(ab, bb, p, s);
+  const int mn = (a_mn ? 1 : 0) | (b_mn ? 2 : 0);
+  switch (mn) {
+    case 0: return p.d_is_bf16 ? launch_gemm2<256, 1, true>(ab, bb, p, s) : launch_gemm2<256, 0, true>(ab, bb, p, s);
+    case 2: return p.d_is_bf16 ? launch_gemm2<256, 1, true, false, 2>(ab, bb, p, s) : launch_gemm2<256, 0, true, false, 2>(ab, bb, p, s);
+    case 3: return p.d_is_bf16 ? launch_gemm2<256, 1, true, false, 3>(ab, bb, p, s) : launch_gemm2<256, 0, true, false, 3>(ab, bb, p, s);
+    default: return NVFP4_ERR_ENUM;
+  }
 }
+}  // namespace
 
 extern "C" int nvfp4_device_error_word(uint32_t* host_out) {
   if (!host_out) return NVFP4_ERR_NULL;

@@ -1,9 +1,9 @@
 // The backward and update products of the paper's quantization-aware fine-tuning phase (Section 5:
 // the forward pass stays in NVFP4, the backward and update GEMMs run in BF16):
 //   dX[M,K] = dY[M,N] . W[N,K]          dW[N,K] = dY[M,N]^T . X[M,K]
-// Both are computed by the bf16 variant of the CTA-pair GEMM, which contracts over the contiguous
-// axis of both operands; the operands that are stored the other way round (W and X for their own
-// products, dY for the update) are transposed first by a tiled bf16 transpose.
+// Both are computed by the bf16 variant of the CTA-pair GEMM.  The operands that are stored with the output
+// axis contiguous (W and X for their own products, dY for the update) are read as they are, through MN-major
+// shared-memory descriptors; nvfp4_transpose_bf16 remains as a utility.
 #include <cuda_bf16.h>
 
 #include "common.cuh"
@@ -70,28 +70,21 @@ extern "C" int nvfp4_transpose_bf16(const void* x, int64_t rows, int64_t cols, i
 }
 
 extern "C" size_t nvfp4_linear_bwd_bf16_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-  if (M <= 0 || N <= 0 || K <= 0) return 0;
-  return align256((size_t)N * K * 2) + align256((size_t)M * K * 2) + align256((size_t)M * N * 2);
+  (void)M; (void)N; (void)K;
+  return 0;                      // the products read W, X and dY as they are stored: nothing is staged
 }
 
 extern "C" int nvfp4_linear_bwd_bf16(const void* dY, const void* W, const void* X, int64_t M, int64_t N, int64_t K,
                                      void* dX, int dx_dtype, void* dW, int dw_dtype,
                                      void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  (void)workspace; (void)workspace_bytes;
   if (!dY || !W || !X || !dX || !dW) return NVFP4_ERR_NULL;
   if ((dx_dtype != NVFP4_BF16 && dx_dtype != NVFP4_FP32) || (dw_dtype != NVFP4_BF16 && dw_dtype != NVFP4_FP32)) return NVFP4_ERR_ENUM;
   if (M <= 0 || N <= 0 || K <= 0 || M % 16 != 0 || N % 16 != 0 || K % 16 != 0) return NVFP4_ERR_SHAPE;
-  const size_t need = nvfp4_linear_bwd_bf16_workspace_bytes(M, N, K);
-  if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 255u)) return NVFP4_ERR_WORKSPACE;
-  uint8_t* ws = static_cast<uint8_t*>(workspace);
-  void* Wt = ws;                                             // [K, N]
-  void* Xt = ws + align256((size_t)N * K * 2);               // [K, M]
-  void* dYt = static_cast<uint8_t*>(Xt) + align256((size_t)M * K * 2);   // [N, M]
-  int st;
-  if ((st = nvfp4_transpose_bf16(W, N, K, K, Wt, cuda_stream))) return st;
-  if ((st = nvfp4_transpose_bf16(X, M, K, K, Xt, cuda_stream))) return st;
-  if ((st = nvfp4_transpose_bf16(dY, M, N, N, dYt, cuda_stream))) return st;
-  // dX[M,K] = dY[M,N] . (W^T)[K,N]^T, contraction over N
-  if ((st = nvfp4_gemm_bf16(dY, Wt, M, K, N, dX, dx_dtype, K, cuda_stream))) return st;
-  // dW[N,K] = (dY^T)[N,M] . (X^T)[K,M]^T, contraction over the token axis M
-  return nvfp4_gemm_bf16(dYt, Xt, N, K, M, dW, dw_dtype, K, cuda_stream);
+  if (!aligned16(dY) || !aligned16(W) || !aligned16(X) || !aligned16(dX) || !aligned16(dW)) return NVFP4_ERR_ALIGN;
+  // dX[M,K] = dY[M,N] . W[N,K]: contraction over N; dY has N contiguous (K-major operand), W is [contraction, output]
+  // with the output axis contiguous (MN-major operand)
+  if (int st = nvfp4_gemm_bf16_ex(dY, 0, W, 1, M, K, N, dX, dx_dtype, K, cuda_stream)) return st;
+  // dW[N,K] = dY[M,N]^T . X[M,K]: contraction over the token axis M; both operands are [contraction, output]
+  return nvfp4_gemm_bf16_ex(dY, 1, X, 1, N, K, M, dW, dw_dtype, K, cuda_stream);
 }

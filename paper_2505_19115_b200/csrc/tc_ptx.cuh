@@ -201,6 +201,14 @@ __device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
   return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) |
          ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
 }
+// The same 128-byte-swizzled rows holding an operand whose OTHER axis is contiguous in memory (MN-major: a row of
+// shared memory is one contraction index and 64 consecutive rows/columns of the output): 8-row groups (8 contraction
+// indices) are 1024 bytes apart (stride offset), successive groups of 64 output rows `mn_chunk_bytes` apart (leading
+// offset).  Only 16-bit operands have this form.
+__device__ __forceinline__ uint64_t operand_desc_mn(uint32_t smem_addr, uint32_t mn_chunk_bytes) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(mn_chunk_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
 // Scale tile: 32 rows x 16 bytes, no swizzle, 8-row groups 128 bytes apart.
 __device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
   return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(128 >> 4) << 32) | ((uint64_t)1 << 46);
@@ -208,8 +216,10 @@ __device__ __forceinline__ uint64_t sf_desc(uint32_t smem_addr) {
 // Instruction descriptor of kind::mxf4nvf4: E2M1 x E2M1 (format 1), K-major operands, UE4M3
 // scales, N >> 3 at bit 17, M >> 4 at bit 24.
 // Instruction descriptor of kind::f16 with bf16 operands (format 1) and an fp32 accumulator (bit 4).
-__host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+// a_mn / b_mn: the operand is MN-major (bits 15 / 16) instead of contiguous along the contraction axis.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int m, int n, bool a_mn = false, bool b_mn = false) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 // Instruction descriptor of kind::mxf4 (scale_vec::2X): as above with UE8M0 scales (bit 23) and the
 // half of the 32-bit scale column to use (bytes 0-1 or 2-3) at bits 4-5 (B) and 29-30 (A).

@@ -158,4 +158,6 @@ def test_newer_entry_points_reject_bad_arguments_on_the_host():
     assert nz(x=None) == 1 and nz(sums=None) == 1 and nz(cols=24) == 2 and nz(sums=C.c_void_p(0x1004)) == 3
     tr = lambda **kw: L.nvfp4_transpose_bf16(kw.get("x", buf), kw.get("rows", 64), 64, 64, buf, None)
     assert tr(x=None) == 1 and tr(rows=60) == 2
-    assert L.nvfp4_linear_bwd_bf16_workspace_bytes(256, 512, 512) > 0 and L.nvfp4_linear_bwd_bf16_workspace_bytes(0, 512, 512) == 0
+    assert L.nvfp4_linear_bwd_bf16_workspace_bytes(256, 512, 512) == 0          # operands are read in place
+    gx = lambda **kw: L.nvfp4_gemm_bf16_ex(kw.get("a", buf), kw.get("am", 0), buf, kw.get("bm", 0), kw.get("M", 128), 128, 64, buf, 1, 128, None)
+    assert gx(a=None) == 1 and gx(am=2) == 4 and gx(am=1, bm=0) == 4 and gx(am=1, bm=1, M=100) == 2
