@@ -11,6 +11,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "quantize_core.cuh"
 #include "tensor_map.cuh"
 
@@ -53,6 +55,25 @@ __device__ __forceinline__ uint32_t swz128(uint32_t row, uint32_t byte) {
 // MX_T: the transposed output is MXFP4 (Section 3, Table 1): blocks of 32 rows with an E8M0 scale rounded up to a
 // power of two; a warp then takes 32 rows at a time, and the two groups of 16 inside a block keep their own
 // random draws (group index as for NVFP4).
+// Shared-memory accesses with the address split into a register part and a compile-time byte offset, so that
+// the unrolled loops below spend no instructions on addresses.
+template <int IMM>
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.b32 %0, [%1 + %2];" : "=r"(v) : "r"(addr), "n"(IMM));
+  return v;
+}
+template <int IMM>
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4 + %5];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr), "n"(IMM));
+  return v;
+}
+template <int IMM>
+__device__ __forceinline__ void sts64(uint32_t addr, uint32_t lo, uint32_t hi) {
+  asm volatile("st.shared.v2.b32 [%0 + %3], {%1, %2};" ::"r"(addr), "r"(lo), "r"(hi), "n"(IMM) : "memory");
+}
+
 template <bool SR_T, bool DUAL, bool SR_R, bool SWZ, bool MX_T = false>
 __global__ void __launch_bounds__(kThreads, 4)
 quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_ct,
@@ -140,57 +161,85 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     sf_t[rb * kTileCols + 2 * lane] = (uint8_t)sfa;
     sf_t[rb * kTileCols + 2 * lane + 1] = (uint8_t)sfb;
   } else {
+  {
+    // Row rb*16 + j of the tile, bytes 4*lane..4*lane+3: (row & 7) = j & 7, so the swizzled position inside a
+    // row depends on j & 7 only; eight base addresses serve all loads, the rest is a compile-time offset.
+    const uint32_t tile_s = smem_addr(tile) + (uint32_t)warp * 2048u;
+    uint32_t rowbase[8];
 #pragma unroll
-  for (int rb = warp; rb < kTileRows / 16; rb += kThreads / 32) {
-    uint32_t w[16];
+    for (int q = 0; q < 8; ++q) rowbase[q] = tile_s + q * 128 + ((((uint32_t)(lane >> 2) ^ q) << 4) | ((uint32_t)(lane & 3) << 2));
+    // staging position of this lane's two output rows (columns 2*lane, 2*lane+1) for row block `warp`; the second
+    // row block of this warp (warp + 8) sits four 16-byte chunks further, which the swizzle turns into an XOR with 64
+    const uint32_t ct_s = smem_addr(codes_t);
+    const uint32_t ra = 2 * lane, rbw = 2 * lane + 1;
+    const uint32_t st_a = ct_s + ra * 128 + ((((uint32_t)(warp >> 1) ^ (ra & 7)) << 4) | ((uint32_t)(warp & 1) << 3));
+    const uint32_t st_b = ct_s + rbw * 128 + ((((uint32_t)(warp >> 1) ^ (rbw & 7)) << 4) | ((uint32_t)(warp & 1) << 3));
+    const uint64_t blk_a0 = (uint64_t)((c0 + 2 * lane) * p.t_nkb + r0 / 16 + warp);
+    uint8_t* sf_lane = sf_t + warp * kTileCols + 2 * lane;
 #pragma unroll
-    for (int j = 0; j < 16; ++j) w[j] = *reinterpret_cast<const uint32_t*>(tile + swz128(rb * 16 + j, 4 * lane));
-    uint32_t m[8];
+    for (int it = 0; it < 2; ++it) {                          // row blocks warp and warp + 8
+      uint32_t w[16];
 #pragma unroll
-    for (int j = 0; j < 8; ++j) m[j] = absmax_bf16x2(w[2 * j], w[2 * j + 1]);
+      for (int j = 0; j < 8; ++j) {
+        w[j] = it ? lds32<16384 + 0>(rowbase[j]) : lds32<0>(rowbase[j]);
+        w[j + 8] = it ? lds32<16384 + 1024>(rowbase[j]) : lds32<1024>(rowbase[j]);
+      }
+      uint32_t m[8];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) m[j] = absmax_bf16x2(m[2 * j], m[2 * j + 1]);
-    const uint32_t mm = absmax_bf16x2(absmax_bf16x2(m[0], m[1]), absmax_bf16x2(m[2], m[3])) & 0x7FFF7FFFu;
-    float va[16], vb[16];
+      for (int j = 0; j < 8; ++j) m[j] = absmax_bf16x2(w[2 * j], w[2 * j + 1]);
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      va[j] = __uint_as_float(w[j] << 16);                    // column 2*lane
-      vb[j] = __uint_as_float(w[j] & 0xFFFF0000u);            // column 2*lane + 1
+      for (int j = 0; j < 4; ++j) m[j] = absmax_bf16x2(m[2 * j], m[2 * j + 1]);
+      const uint32_t mm = absmax_bf16x2(absmax_bf16x2(m[0], m[1]), absmax_bf16x2(m[2], m[3])) & 0x7FFF7FFFu;
+      float va[16], vb[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        va[j] = __uint_as_float(w[j] << 16);                  // column 2*lane
+        vb[j] = __uint_as_float(w[j] & 0xFFFF0000u);          // column 2*lane + 1
+      }
+      const uint64_t blk_a = blk_a0 + 8u * it, blk_b = blk_a + (uint64_t)p.t_nkb;
+      uint32_t lo, hi, sfa, sfb;
+      encode_block<SR_T>(va, __uint_as_float(mm << 16), c, inv_table, p.t_rng, blk_a, lo, hi, sfa);
+      if (it) sts64<0>(st_a ^ 64u, lo, hi); else sts64<0>(st_a, lo, hi);
+      encode_block<SR_T>(vb, __uint_as_float(mm & 0xFFFF0000u), c, inv_table, p.t_rng, blk_b, lo, hi, sfb);
+      if (it) sts64<0>(st_b ^ 64u, lo, hi); else sts64<0>(st_b, lo, hi);
+      *reinterpret_cast<uint16_t*>(sf_lane + it * 8 * kTileCols) = (uint16_t)(sfa | (sfb << 8));
     }
-    const int64_t kb = r0 / 16 + rb;
-    const int64_t ca = c0 + 2 * lane;
-    uint32_t lo, hi, sf;
-    encode_block<SR_T>(va, __uint_as_float(mm << 16), c, inv_table, p.t_rng, (uint64_t)(ca * p.t_nkb + kb), lo, hi, sf);
-    *reinterpret_cast<uint2*>(codes_t + swz128(2 * lane, rb * 8)) = make_uint2(lo, hi);
-    sf_t[rb * kTileCols + 2 * lane] = (uint8_t)sf;
-    encode_block<SR_T>(vb, __uint_as_float(mm & 0xFFFF0000u), c, inv_table, p.t_rng, (uint64_t)((ca + 1) * p.t_nkb + kb), lo, hi, sf);
-    *reinterpret_cast<uint2*>(codes_t + swz128(2 * lane + 1, rb * 8)) = make_uint2(lo, hi);
-    sf_t[rb * kTileCols + 2 * lane + 1] = (uint8_t)sf;
   }
   }
 
   // ---- row output: thread -> (row, block of 16 columns); four rows per thread ----
   if constexpr (DUAL) {
     const int kbl = threadIdx.x & 3;                          // block within the tile's 64 columns
-#pragma unroll 1
-    for (int i = 0; i < kTileRows / 64; ++i) {
-      const int rl = i * 64 + (threadIdx.x >> 2);
-      const uint4 a = *reinterpret_cast<const uint4*>(tile + swz128(rl, kbl * 32));
-      const uint4 b = *reinterpret_cast<const uint4*>(tile + swz128(rl, kbl * 32 + 16));
+    const int t = threadIdx.x >> 2;                           // row within a group of 64; (row & 7) = t & 7 for all four groups
+    const uint32_t ld_a = smem_addr(tile) + (uint32_t)t * 128u + (((uint32_t)(2 * kbl) ^ (uint32_t)(t & 7)) << 4);
+    const uint32_t ld_b = ld_a ^ 16u;                         // the neighbouring 16-byte chunk
+    const uint32_t st_r = smem_addr(codes_r) + (uint32_t)t * 32u + (uint32_t)kbl * 8u;
+    uint8_t* sf_thread = sf_r + (t & 31) * 16 + (t >> 5) * 4 + kbl;
+    const uint64_t blk_r0 = (uint64_t)((r0 + t) * p.r_nkb + c0 / 16 + kbl);
+    const uint64_t blk_step = (uint64_t)(64 * p.r_nkb);
+    auto row_block = [&](auto I) {
+      constexpr int i = decltype(I)::value;
+      const uint4 a = lds128<i * 8192>(ld_a);
+      const uint4 b = lds128<i * 8192>(ld_b);
       Block16<__nv_bfloat16> blk;
       blk.w[0] = a.x; blk.w[1] = a.y; blk.w[2] = a.z; blk.w[3] = a.w;
       blk.w[4] = b.x; blk.w[5] = b.y; blk.w[6] = b.z; blk.w[7] = b.w;
       float v[16];
       const float amax = blk.unpack(v);
       uint32_t lo, hi, sf;
-      encode_block<SR_R>(v, amax, c, inv_table, p.r_rng, (uint64_t)((r0 + rl) * p.r_nkb + c0 / 16 + kbl), lo, hi, sf);
-      *reinterpret_cast<uint2*>(codes_r + rl * 32 + kbl * 8) = make_uint2(lo, hi);
+      encode_block<SR_R>(v, amax, c, inv_table, p.r_rng, blk_r0 + (uint64_t)i * blk_step, lo, hi, sf);
+      sts64<i * 2048>(st_r, lo, hi);
       if constexpr (SWZ) {
-        sf_r[(rl >> 7) * 512 + (rl & 31) * 16 + ((rl >> 5) & 3) * 4 + kbl] = (uint8_t)sf;
+        sf_thread[(i >> 1) * 512 + (i & 1) * 8] = (uint8_t)sf;
       } else {
+        const int rl = i * 64 + t;
         if (r0 + rl < p.rows && c0 / 16 + kbl < p.r_nkb) p.r_scales[(r0 + rl) * p.r_nkb + c0 / 16 + kbl] = (uint8_t)sf;
       }
-    }
+    };
+    row_block(std::integral_constant<int, 0>{});
+    row_block(std::integral_constant<int, 1>{});
+    row_block(std::integral_constant<int, 2>{});
+    row_block(std::integral_constant<int, 3>{});
   }
 
   // ---- codes out: tiled bulk stores from the staging buffers (clipped at the tensor edge) ----
