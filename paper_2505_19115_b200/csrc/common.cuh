@@ -156,4 +156,23 @@ __device__ __forceinline__ uint4 philox4x32_10(const PhiloxStream& s, uint32_t c
   return make_uint4(c0, c1, c2, c3);
 }
 
+// Two independent calls with their rounds interleaved (two dependency chains in flight per thread).
+__device__ __forceinline__ void philox4x32_10_x2(const PhiloxStream& s, uint64_t blk_a, uint64_t blk_b, uint4& ra, uint4& rb) {
+  uint32_t a0 = (uint32_t)blk_a, a1 = (uint32_t)(blk_a >> 32), a2 = s.off_lo, a3 = s.off_hi;
+  uint32_t b0 = (uint32_t)blk_b, b1 = (uint32_t)(blk_b >> 32), b2 = s.off_lo, b3 = s.off_hi;
+#pragma unroll
+  for (int i = 0; i < 10; ++i) {
+    const uint64_t pa0 = (uint64_t)a0 * 0xD2511F53ull, pa1 = (uint64_t)a2 * 0xCD9E8D57ull;
+    const uint64_t pb0 = (uint64_t)b0 * 0xD2511F53ull, pb1 = (uint64_t)b2 * 0xCD9E8D57ull;
+    a0 = (uint32_t)(pa1 >> 32) ^ a1 ^ s.k0[i];
+    b0 = (uint32_t)(pb1 >> 32) ^ b1 ^ s.k0[i];
+    a2 = (uint32_t)(pa0 >> 32) ^ a3 ^ s.k1[i];
+    b2 = (uint32_t)(pb0 >> 32) ^ b3 ^ s.k1[i];
+    a1 = (uint32_t)pa1; a3 = (uint32_t)pa0;
+    b1 = (uint32_t)pb1; b3 = (uint32_t)pb0;
+  }
+  ra = make_uint4(a0, a1, a2, a3);
+  rb = make_uint4(b0, b1, b2, b3);
+}
+
 }  // namespace nvfp4
