@@ -1,15 +1,18 @@
 // Block-scaled NVFP4 GEMM on the 5th-generation tensor cores (the contraction of Eq. 1-3):
 //   D[m,n] = (gA*gB) * sum_kb sA[m,kb]*sB[n,kb] * sum_{k in kb} a[m,k]*b[n,k]
 //
-// One persistent CTA per SM, warp-specialised:
-//   warp 0      TMA producer: packed codes by tiled bulk-tensor copies (128-byte swizzle), scale
-//               tiles by plain bulk copies, into a ring of shared-memory stages
-//   warp 1      MMA issuer: copies the stage's scales to tensor memory (tcgen05.cp) and issues
-//               tcgen05.mma kind::mxf4nvf4 (128 x BN x 64 per instruction), fp32 accumulators
-//               in tensor memory, double-buffered so the epilogue of tile i overlaps tile i+1
-//   warps 2..5  epilogue: tcgen05.ld the accumulator, scale by gA*gB, store fp32 or bf16
-// Every wait on an mbarrier is bounded in time; on a timeout the CTA records the site in a device
-// error word, drains its outstanding copies, frees its tensor memory and returns.
+// Two kernels, both persistent and warp-specialised, both with every mbarrier wait bounded in time (on a timeout the
+// CTA records the site in a device error word, gives its outstanding copies time to land, frees its tensor memory
+// and returns):
+//
+//   gemm2_nvfp4_kernel   the product kernel: a cluster of two CTAs computes a 256 x 256 tile with
+//                        tcgen05.mma.cta_group::2 (described above its definition); variants for bf16 / fp32 /
+//                        quantized output, MXFP4 operands, bf16 operands (K-major or read in place MN-major)
+//   gemm_nvfp4_kernel    the first design, one CTA per tile (128 x BN): warp 0 stages packed codes by tiled bulk
+//                        copies and scale tiles by plain bulk copies, warp 1 copies the stage's scales to tensor
+//                        memory with tcgen05.cp and issues 128 x BN x 64 MMAs into double-buffered accumulators,
+//                        warps 2-5 read the accumulator out.  Kept as an independent second implementation that the
+//                        tests compare the product kernel with, bit for bit.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
