@@ -4,6 +4,8 @@
 // per-tensor amax scale.  All kernels are HBM-bound streaming kernels.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "quantize_core.cuh"
 
 namespace nvfp4 {
@@ -49,6 +51,11 @@ __global__ void __launch_bounds__(kThreads, 3) quantize_row_kernel(const QuantPa
   __syncthreads();
 
   constexpr int U = (sizeof(T) == 2) ? 4 : 2;  // rows in flight per thread (32 packed registers)
+  // A CTA whose 128 x 512 tile lies wholly inside the tensor (all of them but the last row and column of the grid)
+  // runs the loop without any per-row or per-block predicate.
+  const bool full_tile = row0 + kRowTileRows <= p.rows && ((int64_t)blockIdx.x + 1) * 32 <= p.nkb;
+  auto sweep = [&](auto full_c) {
+  constexpr bool FULL = decltype(full_c)::value;
 #pragma unroll 1
   for (int it = 0; it < kRowTileRows / 8; it += U) {
     Block16<T> raw[U];
@@ -56,7 +63,7 @@ __global__ void __launch_bounds__(kThreads, 3) quantize_row_kernel(const QuantPa
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const int64_t r = row0 + warp + 8 * (it + u);
-      ok[u] = kb_ok && r < p.rows;
+      ok[u] = FULL || (kb_ok && r < p.rows);
       if (ok[u]) raw[u].load(x + r * p.ld + kb * 16, aligned32);
     }
 #pragma unroll
@@ -85,6 +92,8 @@ __global__ void __launch_bounds__(kThreads, 3) quantize_row_kernel(const QuantPa
       }
     }
   }
+  };
+  if (full_tile) sweep(std::true_type{}); else sweep(std::false_type{});
 
   if constexpr (SWZ) {
     __syncthreads();
