@@ -188,3 +188,32 @@ def test_quantizer_sweep_at_2p28_elements():
         _assert_operand_bytes(ct, s_t, *want[("t", k_t)], f"dual transposed {k_t}")
         del cr, s_r, ct, s_t
     assert nb.nvfp4_device_error_word() == 0
+
+
+def test_chained_up_and_down_projection_at_llama7b_size():
+    # the chain bench.py times: the up projection's product leaves its GEMM quantized (nvfp4_linear_fwd_qout) and feeds
+    # the down projection (nvfp4_linear_fwd_qin).  The fp32 product of the same layer is sampled against the oracle; the
+    # quantized product must then be the oracle's quantization of that fp32 product over the whole tensor, byte for
+    # byte, and the second product the oracle's product of those codes at the sampled positions.
+    M, K1, N1, N2 = synth.LLAMA_7B["tokens"], 4096, 11008, 4096
+    X, W1, _ = synth.linear_inputs(M, K1, N1, seed=1021, device="cuda")
+    _, W2, _ = synth.linear_inputs(M, N1, N2, seed=1022, device="cuda")
+    rt = nb.Rounding(nb.RTN)
+    rng = np.random.default_rng(1021)
+    H = nb.nvfp4_linear_fwd(X, W1, rx=rt, rw=rt)
+    hX, hW1 = _host(X), _host(W1)
+    (gx_t, gx), (g1_t, g1) = _scale(X, hX), _scale(W1, hW1)
+    _assert_product(H, _oq(hX, gx, rt), _oq(hW1, g1, rt), gx, g1, rng, "H", (_MIDS[M], _MIDS[N1]))
+    del hX, hW1
+    hH = H.cpu().numpy()
+    gh_t, gh = _scale(H, hH)
+    hc, hs = nb.nvfp4_linear_fwd_qout(X, W1, gy=gh_t, ry=rt, rx=rt, rw=rt, sf_layout=nb.SF_SWIZZLED)
+    Y = nb.nvfp4_linear_fwd_qin(hc, hs, gh_t, W2, rw=rt)
+    torch.cuda.synchronize()
+    assert nb.nvfp4_device_error_word() == 0
+    qH = _oq(hH, gh, rt)
+    del hH
+    _assert_operand_bytes(hc, hs, *qH, "Q(H) from the GEMM epilogue")
+    hW2 = _host(W2)
+    g2_t, g2 = _scale(W2, hW2)
+    _assert_product(Y, qH, _oq(hW2, g2, rt), gh, g2, rng, "Y", (_MIDS[M], _MIDS[N2]))
